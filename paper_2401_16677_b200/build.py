@@ -57,11 +57,24 @@ def _compile(out: str, extra, verbose: bool) -> None:
     os.replace(tmp, out)
 
 
+def _multi_process_launch() -> bool:
+    for key in ("WORLD_SIZE", "LOCAL_WORLD_SIZE"):
+        try:
+            if int(os.environ.get(key, "1")) > 1:
+                return True
+        except ValueError:
+            return True
+    return False
+
+
 def build(force: bool = False, verbose: bool = False) -> str:
-    """Builds what is stale (everything with force); returns the path of the portable library."""
+    """Builds what is stale (everything with force); returns the path of the portable library.
+    A rank of a multi-process launch builds (and later loads) the portable library only."""
     deps = [os.path.join(CSRC, d) for d in DEPS]
     if force or _stale(LIB, deps):
         _compile(LIB, [], verbose)
+    if _multi_process_launch():
+        return LIB
     if os.path.exists(SHARED_FETCH_SRC):
         if force or _stale(LIB_SF, deps + [SHARED_FETCH_SRC]):
             _compile(LIB_SF, ["-DT3_TMA_SHARED_FETCH"], verbose)

@@ -1,8 +1,12 @@
 """ctypes binding of the C-ABI library (declared in include/t3.h).
 
 The build makes ``libt3.so`` and, where its extra source file is present,
-``libt3_sf.so`` (same ABI plus the 4-CTA-cluster kernel variant); the binding
-loads the latter when it exists.  ``T3_LIB_PATH`` overrides the choice.
+``libt3_sf.so`` (same ABI plus the 4-CTA-cluster kernel variant, whose W
+fetches are TMA loads multicast to two CTA pairs).  That variant is for
+single-process, single-GPU use only: the binding loads it when it exists AND
+the process is not part of a multi-process launch (``WORLD_SIZE`` or
+``LOCAL_WORLD_SIZE`` above 1); in such a launch it always loads ``libt3.so``,
+whatever files exist and whatever ``T3_LIB_PATH`` says about the variant.
 
 Argument marshalling only: every step of the path runs in the library's CUDA
 kernels.  Function names mirror the C names without the ``t3_`` prefix.
@@ -16,8 +20,34 @@ import os
 from typing import List, Optional, Tuple
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PORTABLE = os.path.join(_HERE, "libt3.so")
 _LIB_SF = os.path.join(_HERE, "libt3_sf.so")
-LIB_PATH = os.environ.get("T3_LIB_PATH") or (_LIB_SF if os.path.exists(_LIB_SF) else os.path.join(_HERE, "libt3.so"))
+
+
+def multi_process_launch(env=None) -> bool:
+    """True when this process is one rank of a launch with more than one process."""
+    env = os.environ if env is None else env
+    for key in ("WORLD_SIZE", "LOCAL_WORLD_SIZE"):
+        try:
+            if int(env.get(key, "1")) > 1:
+                return True
+        except ValueError:
+            return True          # unreadable: assume the cautious answer
+    return False
+
+
+def choose_lib_path(env=None) -> str:
+    """The library this process may load.  The multicast variant is never chosen in a multi-process launch."""
+    env = os.environ if env is None else env
+    if multi_process_launch(env):
+        return _LIB_PORTABLE
+    override = env.get("T3_LIB_PATH")
+    if override:
+        return override
+    return _LIB_SF if os.path.exists(_LIB_SF) else _LIB_PORTABLE
+
+
+LIB_PATH = choose_lib_path()
 
 OK = 0
 ERR_INVALID_ARG, ERR_SHAPE, ERR_DEVICE, ERR_ALLOC, ERR_CUDA, ERR_TIMEOUT, ERR_UNSUPPORTED, ERR_TOO_LARGE = \

@@ -3,6 +3,7 @@ validation, plan geometry, producer schedule, tracker thresholds, ring order."""
 import ctypes
 import os
 import re
+import sys
 from collections import Counter
 
 import pytest
@@ -253,3 +254,27 @@ def test_plan_without_gpu_fails_loudly():
     assert e.value.code == t3.ERR_DEVICE
     assert t3.lib().t3_gemm_rs(None, None, None, None, None) == t3.ERR_INVALID_ARG
     assert t3.lib().t3_destroy(None) == 0
+
+
+def test_multicast_variant_is_never_chosen_in_a_multi_process_launch():
+    """The library variant with the multicast W fetch is for one process on one GPU: any launch with
+    WORLD_SIZE or LOCAL_WORLD_SIZE above 1 gets the portable library, whatever files exist and whatever
+    T3_LIB_PATH asks for."""
+    here = os.path.dirname(os.path.abspath(t3.__file__))
+    portable = os.path.join(here, "libt3.so")
+    sf = os.path.join(here, "libt3_sf.so")
+    for env in ({"WORLD_SIZE": "2"}, {"LOCAL_WORLD_SIZE": "8"}, {"WORLD_SIZE": "2", "T3_LIB_PATH": sf},
+                {"WORLD_SIZE": "junk"}):
+        assert t3.multi_process_launch(env)
+        assert t3.choose_lib_path(env) == portable, env
+    assert not t3.multi_process_launch({"WORLD_SIZE": "1"})
+    assert not t3.multi_process_launch({})
+    assert t3.choose_lib_path({"T3_LIB_PATH": "/x/y.so"}) == "/x/y.so"
+    # a fresh interpreter started as rank 0 of 2 binds the portable library
+    import subprocess
+    env = dict(os.environ, WORLD_SIZE="2", RANK="0")
+    env.pop("T3_LIB_PATH", None)
+    out = subprocess.check_output([sys.executable, "-c",
+                                   "from paper_2401_16677_b200 import t3; print(t3.LIB_PATH); "
+                                   "print(t3.shared_fetch_available())"], cwd=ROOT, env=env, text=True).split()
+    assert out[0] == portable and out[1] == "False"
