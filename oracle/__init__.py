@@ -6,6 +6,8 @@ from .t3_oracle import (  # noqa: F401
     ring_order,
     ring_sum_f32,
     chunks,
+    epilogue,
+    epilogue_f32,
     threads,
     max_rel_err,
 )

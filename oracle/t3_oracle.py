@@ -127,6 +127,40 @@ def ring_sum_f32(P: np.ndarray) -> np.ndarray:
     return Y
 
 
+def epilogue(Y: np.ndarray, bias: Optional[np.ndarray] = None, keep: Optional[np.ndarray] = None,
+             keep_scale: float = 1.0, residual: Optional[np.ndarray] = None) -> np.ndarray:
+    """The element-wise operators that follow the all-reduce, applied to the reduced array (Section 7.6:
+    bias, dropout and residual add can run on each device's reduce-scattered chunk before the all-gather):
+
+        out[m][n] = (Y[m][n] + bias[n]) * (keep_scale if keep[m][n] else 0) + residual[m][n]
+
+    in fp64.  The dropout mask is an input (whoever drew it); a missing operand skips its step.
+    Y [rows,N]; bias [N]; keep, residual [rows,N] (the same rows as Y)."""
+    out = np.array(Y, dtype=np.float64, copy=True)
+    if bias is not None:
+        out = out + np.asarray(bias, dtype=np.float64)[None, :]
+    if keep is not None:
+        out = out * np.where(np.asarray(keep) != 0, np.float64(keep_scale), np.float64(0.0))
+    if residual is not None:
+        out = out + np.asarray(residual, dtype=np.float64)
+    return out
+
+
+def epilogue_f32(S: np.ndarray, bias: Optional[np.ndarray] = None, keep: Optional[np.ndarray] = None,
+                 keep_scale: float = 1.0, residual: Optional[np.ndarray] = None) -> np.ndarray:
+    """The same three steps in device arithmetic: each one a single fp32 operation rounded to nearest
+    (add, multiply, add; nothing fused), on an fp32 sum S.  Lets a test check the fused tail bit for bit
+    given the device's own reduced sum."""
+    out = np.array(S, dtype=np.float32, copy=True)
+    if bias is not None:
+        out = (out + np.asarray(bias, dtype=np.float32)[None, :]).astype(np.float32)
+    if keep is not None:
+        out = (out * np.where(np.asarray(keep) != 0, np.float32(keep_scale), np.float32(0.0))).astype(np.float32)
+    if residual is not None:
+        out = (out + np.asarray(residual, dtype=np.float32)).astype(np.float32)
+    return out
+
+
 def chunks(Y: np.ndarray, R: int) -> List[np.ndarray]:
     """Reduce-scatter view (Section 2.3): chunk c = rows [c*M/R, (c+1)*M/R),
     the part device c owns after the collective."""

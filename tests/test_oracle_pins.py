@@ -370,3 +370,61 @@ def test_sample_rows_cover_chunks():
     for c in range(16):
         assert c * cr in rows and (c + 1) * cr - 1 in rows
     assert len(rows) <= 4096 // 16 + 32
+
+
+# ---------------------------------------------------------------------------
+# the element-wise tail on the reduced chunk (Section 7.6): bias, dropout mask, residual
+# ---------------------------------------------------------------------------
+
+def test_epilogue_closed_forms():
+    """All-ones inputs with a constant bias give K + b everywhere; a dropped element is exactly the
+    residual; a kept one is (K + b) * scale + residual.  A wrong order of the three steps (bias after the
+    mask, residual before it) or a mask applied to the residual changes these values."""
+    M, N, K, R = 8, 16, 32, 4
+    ones = wl.f32_to_bf16_bits(np.ones((M, K), dtype=np.float32))
+    wones = wl.f32_to_bf16_bits(np.ones((K, N), dtype=np.float32))
+    Y = oracle.gemm_rs(ones, wones, R)
+    assert np.all(Y == K)
+    b = np.full(N, 0.5)
+    assert np.all(oracle.epilogue(Y, bias=b) == K + 0.5)
+    keep = np.zeros((M, N), dtype=np.uint8)
+    keep[::2] = 1
+    res = np.full((M, N), 3.0)
+    out = oracle.epilogue(Y, bias=b, keep=keep, keep_scale=2.0, residual=res)
+    assert np.all(out[::2] == (K + 0.5) * 2.0 + 3.0)
+    assert np.all(out[1::2] == 3.0)
+    # bias is per column, the mask and the residual per element
+    b2 = np.arange(N, dtype=np.float64)
+    out2 = oracle.epilogue(Y, bias=b2)
+    assert np.array_equal(out2, K + np.tile(b2, (M, 1)))
+    # no operand: identity
+    assert np.array_equal(oracle.epilogue(Y), Y)
+
+
+def test_epilogue_residual_cancels_the_product_exactly():
+    """residual = -(X.W) on exact-integer inputs leaves exactly zero (the reduced sum and the residual
+    meet with opposite signs: a sign slip or a dropped slice leaves a non-zero)."""
+    M, N, K, R = 12, 24, 64, 4
+    xb, wb = wl.make_small_int_inputs(M, N, K, seed=9)
+    x = wl.bf16_bits_to_f64(xb).astype(np.int64)
+    w = wl.bf16_bits_to_f64(wb).astype(np.int64)
+    out = oracle.epilogue(oracle.gemm_rs(xb, wb, R), residual=-(x @ w).astype(np.float64))
+    assert np.all(out == 0.0)
+    # the fp32 restatement agrees on exactly representable values
+    s32 = oracle.gemm_rs(xb, wb, R).astype(np.float32)
+    keep = (np.arange(M * N).reshape(M, N) % 3 != 0).astype(np.uint8)
+    b = np.arange(N, dtype=np.float32) - 7
+    r32 = np.arange(M * N, dtype=np.float32).reshape(M, N) % 11
+    got = oracle.epilogue_f32(s32, bias=b, keep=keep, keep_scale=2.0, residual=r32)
+    assert got.dtype == np.float32
+    assert np.array_equal(got.astype(np.float64), oracle.epilogue(s32.astype(np.float64), bias=b, keep=keep, keep_scale=2.0, residual=r32))
+
+
+def test_epilogue_f32_rounds_every_step():
+    """(1e8 + 1) * 1 - 1e8 is 0 when the add is rounded to fp32 before the next step, 1 in fp64."""
+    S = np.array([[1e8]], dtype=np.float32)
+    out32 = oracle.epilogue_f32(S, bias=np.array([1.0]), keep=np.array([[1]], dtype=np.uint8), keep_scale=1.0,
+                                residual=np.array([[-1e8]]))
+    out64 = oracle.epilogue(S.astype(np.float64), bias=np.array([1.0]), keep=np.array([[1]], dtype=np.uint8), keep_scale=1.0,
+                            residual=np.array([[-1e8]]))
+    assert out32[0, 0] == 0.0 and out64[0, 0] == 1.0
