@@ -3,8 +3,11 @@
 
 A "step" is one pass of the whole hot path over one synthetic batch: the
 fused kernel (producer GEMM per K-slice, partial stores, tracker, triggered
-ring-order reduction) on the GPT-2-XL-like FC-2 sublayer (R=8, M=8192,
-K=6400, N=1600) unless --workload says otherwise.
+ring-order reduction) on the largest single-GPU configuration, the large-model
+FC-2 sublayer (R=16, M=4096, K=32768, N=8192, bf16 output), unless --workload
+says otherwise.  The same JSON line carries `per_config`: the other
+configurations (tiny, GPT-2-XL-like FC-2, Mega-GPT-like attention-out and
+FC-2, the large FC-2 with fp32 output) with the four modes timed interleaved.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME]
   python bench.py --impl reference ...      # the CPU oracle on the host cores
@@ -29,14 +32,19 @@ if ROOT not in sys.path:
 
 METRIC = "fused_gemm_rs_tflops"
 UNIT = "TFLOP/s"
-DEFAULT_WORKLOAD = "C2_gpt2xl_fc2"
+DEFAULT_WORKLOAD = "C4_large_fc2"
 L2_FLUSH_BYTES = 512 << 20
 
-# DRAM traffic of one fused-kernel launch measured by ncu (dram__bytes_read.sum +
-# dram__bytes_write.sum); see profiles/.  None until a capture exists for the workload.
-NCU_TRAFFIC_BYTES = {
-    "C2_gpt2xl_fc2": 727.6e6,   # fused-kernel capture summarised under profiles/
+# DRAM traffic of one fused-kernel launch (dram__bytes_read.sum + dram__bytes_write.sum) as captured by
+# ncu in an EARLIER, separate run (never measured inside this script): bytes per launch and the summary
+# under profiles/ that holds the capture's command and figures.  Absent: no capture for that workload.
+NCU_TRAFFIC = {
+    "C2_gpt2xl_fc2": (727.6e6, "profiles/t3_fused_kernel_C2.md"),
+    "C3b_megagpt_fc2": (1286.0e6, "profiles/t3_fused_kernel_C3b.md"),
 }
+CHUNK_ARGS = ("tile_n", "group_tiles", "reducer_ctas", "reducer_warps", "reduce_rows", "stages", "ring_slots", "cluster_ctas",
+              "partial_dtype", "order", "reduce", "split_k")
+PER_CONFIG = ["C1_tiny", "C2_gpt2xl_fc2", "C3a_megagpt_attn_out", "C3b_megagpt_fc2", "C4_large_fc2:f32"]
 
 
 def _peaks():
@@ -213,6 +221,103 @@ def _whole_job_value(world: int, flops_per_replica: float, ms_per_step: float) -
     return world * flops_per_replica / (ms_per_step * 1e-3) / 1e12
 
 
+MODE_NAMES = ("fused", "sequential", "gemm_only", "reduce_only")
+
+
+def _interleaved(torch, t3, plan, X, W, Y, st, flush, rounds, per_round):
+    """The four modes timed round-robin on one plan (same tile shape, schedule and workspace), L2 flushed
+    before every call: `rounds` rounds of `per_round` calls per mode.  Returns per mode the list of
+    per-round medians in microseconds, and the fused kernel's timeline medians."""
+    modes = (t3.MODE_FUSED, t3.MODE_SEQUENTIAL, t3.MODE_GEMM_ONLY, t3.MODE_REDUCE_ONLY)
+    for m in (t3.MODE_GEMM_ONLY,) + modes:       # reduce-only needs valid partial tiles; then one warm call each
+        flush.zero_()
+        plan.gemm_rs_mode(m, X.data_ptr(), W.data_ptr(), Y.data_ptr(), st)
+    torch.cuda.synchronize()
+    us = {n: [] for n in MODE_NAMES}
+    tl = {"produce_us": [], "tail_us": [], "drain_us": [], "total_us": []}
+    for _ in range(rounds):
+        for name, m in zip(MODE_NAMES, modes):
+            ms = _time_mode(torch, plan, m, X, W, Y, st, per_round, 0, flush)
+            us[name].append(1e3 * statistics.median(ms))
+            if m == t3.MODE_FUSED:
+                t = plan.timeline()
+                for k in tl:
+                    tl[k].append(getattr(t, k))
+    return us, {k: statistics.median(v) for k, v in tl.items()}
+
+
+def _overlap_figures(us, timeline):
+    """Exposed / hidden reduction from the per-round medians (Section 5.1.3's configurations: Sequential,
+    and the ideal overlap max(GEMM, RS))."""
+    med = statistics.median
+    f, q, g, r = (med(us[n]) for n in MODE_NAMES)
+    per_round_hidden = [1.0 - max(0.0, fi - gi) / ri for fi, gi, ri in zip(us["fused"], us["gemm_only"], us["reduce_only"])]
+    after_last_tile = timeline["tail_us"] + timeline["drain_us"]
+    return {
+        "us": {"fused": round(f, 2), "sequential": round(q, 2), "gemm_only": round(g, 2), "reduce_only": round(r, 2)},
+        "seq_over_fused": round(q / f, 4),
+        # definition 1: against the GEMM-only MODE (which writes full partial buffers to DRAM)
+        "exposed_reduce_us": round(max(0.0, f - g), 2),
+        "hidden_reduce_frac": round(1.0 - max(0.0, f - g) / r, 4),
+        "hidden_reduce_frac_range": [round(min(per_round_hidden), 4), round(max(per_round_hidden), 4)],
+        # against the ideal overlap of Section 5.1.3: max(GEMM, reduction), no contention
+        "ideal_overlap_us": round(max(g, r), 2),
+        "exposed_vs_ideal_us": round(f - max(g, r), 2),
+        # definition 2: inside the fused kernel itself - what is left after its last partial tile landed
+        "fused_timeline_us": {k.replace("_us", ""): round(v, 2) for k, v in timeline.items()},
+        "exposed_after_last_tile_us": round(after_last_tile, 2),
+        "hidden_after_last_tile_frac": round(1.0 - after_last_tile / r, 4),
+    }
+
+
+def _roofline(info, avg_s, peaks, workload_name):
+    t_flop = info.flops / (peaks["bf16_tflops"] * 1e12)
+    t_byte = info.bytes_fused / (peaks["hbm_gbs"] * 1e9)
+    bound = "hbm" if t_byte >= t_flop else "tensor"
+    if bound == "hbm":
+        achieved, peak, runit = info.bytes_fused / avg_s / 1e9, peaks["hbm_gbs"], "GB/s"
+    else:
+        achieved, peak, runit = info.flops / avg_s / 1e12, peaks["bf16_tflops"], "TFLOP/s"
+    traffic, source = NCU_TRAFFIC.get(workload_name, (None, None))
+    return {
+        "bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
+        "traffic": traffic,
+        "traffic_source": (source + " (ncu capture of an earlier run of this kernel, not measured in this run)") if source else None,
+        "peak_source": peaks["source"] + " (burst figure: each step is one kernel timed alone between L2 flushes)",
+        "kernel": "t3_fused_kernel", "algorithmic_bytes": info.bytes_fused, "flops": info.flops,
+        "t_roof_us": 1e6 * max(t_flop, t_byte),
+        "tensor_frac_of_burst": info.flops / avg_s / 1e12 / peaks["bf16_tflops"],
+        "tensor_frac_of_sustained": info.flops / avg_s / 1e12 / peaks["bf16_tflops_sustained"],
+        "hbm_frac_by_algorithmic_bytes": info.bytes_fused / avg_s / 1e9 / peaks["hbm_gbs"],
+    }
+
+
+def _per_config(torch, np, t3, wl, spec, st, flush, peaks, rounds, per_round):
+    """One entry of the per_config list: a whole configuration, default chunking, four modes interleaved."""
+    name, _, out = spec.partition(":")
+    w = wl.by_name(name)
+    dtype = t3.BF16_OUT_F32 if out == "f32" else t3.BF16_OUT_BF16
+    xb, wb = wl.make_inputs(w)
+    X = torch.from_numpy(xb.view(np.int16)).cuda()
+    W = torch.from_numpy(wl.w_nk(wb).view(np.int16)).cuda()
+    del xb, wb
+    Y = torch.zeros((w.M, w.N), dtype=torch.float32 if dtype == t3.BF16_OUT_F32 else torch.bfloat16, device="cuda")
+    plan = t3.Plan(w.M, w.N, w.K, w.R, dtype, None)
+    info = plan.info()
+    us, tl = _interleaved(torch, t3, plan, X, W, Y, st, flush, rounds, per_round)
+    plan.destroy()
+    entry = {"workload": w.name, "out": out or "bf16", "M": w.M, "N": w.N, "K": w.K, "R": w.R,
+             "tile": [info.tile_m, info.tile_n], "cluster_ctas": info.cluster_ctas, "ring_slots": info.ring_slots}
+    entry.update(_overlap_figures(us, tl))
+    fused_s = entry["us"]["fused"] * 1e-6
+    roof = _roofline(info, fused_s, peaks, w.name)
+    entry["fused_tflops"] = round(info.flops / fused_s / 1e12, 1)
+    entry["roofline"] = {k: roof[k] for k in ("bound", "achieved", "peak", "unit", "frac", "t_roof_us", "traffic", "traffic_source")}
+    del X, W, Y
+    torch.cuda.empty_cache()
+    return entry
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -226,6 +331,10 @@ def run_ours(args):
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     if not torch.cuda.is_available():
         raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback for the product path")
+    if world > 1 and args.cluster_ctas == 4:
+        raise SystemExit("--cluster-ctas 4 is for one process on one GPU (its W fetches are multicast TMA loads)")
+    if world > 1:
+        assert t3.LIB_PATH.endswith("libt3.so"), t3.LIB_PATH
     torch.cuda.set_device(local_rank)
     dist = None
     if world > 1:
@@ -247,12 +356,15 @@ def run_ours(args):
     st = torch.cuda.current_stream().cuda_stream
     flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device="cuda")
     ch_kw = {}
-    for k in ("tile_n", "group_tiles", "reducer_ctas", "reducer_warps", "reduce_rows", "stages", "ring_slots", "cluster_ctas",
-              "partial_dtype", "order"):
+    for k in CHUNK_ARGS:
         v = getattr(args, k)
         if v is not None:
             ch_kw[k] = v
     plan = t3.Plan(w.M, w.N, w.K, w.R, dtype, t3.chunking(**ch_kw) if ch_kw else None)
+    tuned = None
+    if args.tune:
+        res = plan.tune(X.data_ptr(), W.data_ptr(), Y.data_ptr(), st)
+        tuned = {"tried": res.n_tried, "chosen": res.candidates()[res.chosen]}
     info = plan.info()
     peaks = _peaks()
 
@@ -275,15 +387,13 @@ def run_ours(args):
     # ---- headline: fused path, inputs resident in HBM, L2 flushed between steps
     barrier()
     sampler.start()
-    ms_fused = _time_mode(torch, plan, t3.MODE_FUSED, X, W, Y, st, args.steps, args.warmup, flush)
-    # companions on the same plan (same tile shape and schedule)
-    side_steps = max(3, min(args.steps, 50))
-    ms_seq = _time_mode(torch, plan, t3.MODE_SEQUENTIAL, X, W, Y, st, side_steps, 3, flush)
-    ms_gemm = _time_mode(torch, plan, t3.MODE_GEMM_ONLY, X, W, Y, st, side_steps, 3, flush)
-    ms_red = _time_mode(torch, plan, t3.MODE_REDUCE_ONLY, X, W, Y, st, side_steps, 3, flush)
-    ms_fused_warm = _time_mode(torch, plan, t3.MODE_FUSED, X, W, Y, st, side_steps, 3, None)
+    ms_fused = _time_mode(torch, plan, plan.info().mode, X, W, Y, st, args.steps, args.warmup, flush)
     sampler.stop()
     barrier()
+    clocks = sampler.summary()
+    # companions on the same plan (same tile shape and schedule), interleaved round-robin
+    us_modes, timeline = _interleaved(torch, t3, plan, X, W, Y, st, flush, args.rounds, args.per_round)
+    ms_fused_warm = _time_mode(torch, plan, t3.MODE_FUSED, X, W, Y, st, max(3, min(args.steps, 20)), 3, None)
 
     total_ms = float(sum(ms_fused))
     total_ms_max = _max_over_ranks(total_ms, dist, "cuda")
@@ -295,6 +405,7 @@ def run_ours(args):
     Wh = torch.from_numpy(wnk.view(np.int16)).pin_memory()
     Yh = torch.empty((w.M, w.N), dtype=Y.dtype).pin_memory()
     e2e_steps = max(3, min(args.steps, 20))
+    plan.gemm_rs(X.data_ptr(), W.data_ptr(), Y.data_ptr(), st)       # the device-resident result to compare with
     for _ in range(2):
         plan.gemm_rs_host(Xh.data_ptr(), Wh.data_ptr(), Yh.data_ptr(), st)
     barrier()
@@ -309,10 +420,16 @@ def run_ours(args):
     e2e_ms_step = _max_over_ranks(e2e_ms, dist, "cuda") / e2e_steps
     e2e_value = _whole_job_value(world, info.flops, e2e_ms_step)
     # the device result must be the one the host got back
-    assert torch.equal(Yh.view(torch.int16 if Y.dtype == torch.bfloat16 else torch.int32).cuda(),
-                       Y.view(torch.int16 if Y.dtype == torch.bfloat16 else torch.int32)), "e2e output differs"
+    ity = torch.int16 if Y.dtype == torch.bfloat16 else torch.int32
+    assert torch.equal(Yh.view(ity).cuda(), Y.view(ity)), "e2e output differs"
     sy = 4 if dtype == t3.BF16_OUT_F32 else 2
     plan.destroy()
+    del Xh, Wh, Yh, X, W, Y
+    torch.cuda.empty_cache()
+
+    per_config = None
+    if world == 1 and not args.no_per_config:
+        per_config = [_per_config(torch, np, t3, wl, spec, st, flush, peaks, args.rounds, args.per_round) for spec in PER_CONFIG]
 
     if rank != 0:
         if dist is not None:
@@ -320,23 +437,9 @@ def run_ours(args):
         return 0
 
     med = statistics.median
-    us_fused, us_seq, us_gemm, us_red = (1e3 * med(ms_fused), 1e3 * med(ms_seq), 1e3 * med(ms_gemm), 1e3 * med(ms_red))
-    exposed = max(0.0, us_fused - us_gemm)
-    hidden = 1.0 - exposed / us_red if us_red > 0 else None
     avg_s = (total_ms / args.steps) * 1e-3
-    t_flop = info.flops / (peaks["bf16_tflops"] * 1e12)
-    t_byte = info.bytes_fused / (peaks["hbm_gbs"] * 1e9)
-    bound = "hbm" if t_byte >= t_flop else "tensor"
-    if bound == "hbm":
-        achieved, peak, runit = info.bytes_fused / avg_s / 1e9, peaks["hbm_gbs"], "GB/s"
-    else:
-        achieved, peak, runit = info.flops / avg_s / 1e12, peaks["bf16_tflops"], "TFLOP/s"
-    roofline = {
-        "bound": bound, "achieved": achieved, "peak": peak, "unit": runit, "frac": achieved / peak,
-        "traffic": NCU_TRAFFIC_BYTES.get(w.name), "peak_source": peaks["source"] + " (burst: each step timed alone)",
-        "kernel": "t3_fused_kernel", "algorithmic_bytes": info.bytes_fused, "flops": info.flops,
-        "t_roof_us": 1e6 * max(t_flop, t_byte), "tensor_frac_of_burst": info.flops / avg_s / 1e12 / peaks["bf16_tflops"],
-    }
+    roofline = _roofline(info, avg_s, peaks, w.name)
+    overlap = _overlap_figures(us_modes, timeline)
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         cpu = _cpu_oracle_sample(w, xb, wb, budget_s=args.cpu_seconds)
@@ -352,18 +455,25 @@ def run_ours(args):
             "gemm_ctas": info.gemm_ctas, "reducer_ctas": info.reducer_ctas, "reducer_warps": info.reducer_warps,
             "stages": info.stages, "ring_slots": info.ring_slots, "cluster_ctas": info.cluster_ctas,
             "reduce_rows": info.reduce_rows, "partials": "bf16" if info.partial_dtype == t3.PARTIAL_BF16 else "f32",
+            "reduce": "in place" if info.reduce == t3.REDUCE_INPLACE else "ring order", "mode": MODE_NAMES[info.mode],
+            "companions": f"four modes interleaved, {args.rounds} rounds x {args.per_round} flushed calls each",
         },
-        "us_per_sublayer": {"fused": us_fused, "fused_min": 1e3 * min(ms_fused), "fused_l2_warm": 1e3 * med(ms_fused_warm),
-                            "sequential": us_seq, "gemm_only": us_gemm, "reduce_only": us_red},
-        "exposed_reduce_us": exposed, "hidden_reduce_frac": hidden,
-        "ideal_overlap_us": max(us_gemm, us_red),
+        "us_per_sublayer": dict(overlap["us"], fused_headline=1e3 * med(ms_fused), fused_min=1e3 * min(ms_fused),
+                                fused_l2_warm=1e3 * med(ms_fused_warm)),
         "roofline": roofline,
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": 2 * w.M * w.K + 2 * w.K * w.N,
                 "d2h_bytes_per_step": sy * w.M * w.N, "ms_per_step": e2e_ms_step,
                 "api": "t3_gemm_rs_host (pinned host buffers)"},
         "gpu_launches": args.steps,
-        "clocks": sampler.summary(),
+        "clocks": clocks,
     }
+    for k in ("seq_over_fused", "exposed_reduce_us", "hidden_reduce_frac", "hidden_reduce_frac_range", "ideal_overlap_us",
+              "exposed_vs_ideal_us", "fused_timeline_us", "exposed_after_last_tile_us", "hidden_after_last_tile_frac"):
+        line[k] = overlap[k]
+    if tuned is not None:
+        line["tuned"] = tuned
+    if per_config is not None:
+        line["per_config"] = per_config
     if cpu is not None:
         line["cpu_baseline"] = cpu
     print(json.dumps(line), flush=True)
@@ -375,7 +485,8 @@ def run_ours(args):
 def run_sweep(args):
     """--sweep: configuration 5 (R x M x H grid, K = 4H) plus C1..C4: per point fused, sequential,
     GEMM-only and reduce-only microseconds, TFLOP/s, roofline fractions and the hidden-reduction
-    fraction, one JSON line each (also checks fused == sequential bit for bit at every point)."""
+    fraction, one JSON line each (also checks fused == sequential bit for bit at every point).
+    With --tune the "fused" column is t3_gemm_rs after t3_plan_tune, whatever mode that chose."""
     import numpy as np
     import torch
 
@@ -401,17 +512,20 @@ def run_sweep(args):
         del xb, wb
         Y = torch.zeros((w.M, w.N), dtype=torch.bfloat16, device="cuda")
         Y2 = torch.zeros_like(Y)
-        ch_kw = {k: getattr(args, k) for k in ("reduce_rows", "ring_slots", "cluster_ctas", "partial_dtype", "order")
-                 if getattr(args, k, None) is not None}
+        ch_kw = {k: getattr(args, k) for k in CHUNK_ARGS if getattr(args, k, None) is not None}
         try:
             plan = t3.Plan(w.M, w.N, w.K, w.R, t3.BF16_OUT_BF16, t3.chunking(**ch_kw) if ch_kw else None)
         except t3.T3Error as e:      # an override that this shape does not admit
             print(json.dumps({"workload": w.name, "skipped": str(e)}), flush=True)
             continue
+        chosen = None
+        if args.tune:
+            res = plan.tune(X.data_ptr(), W.data_ptr(), Y.data_ptr(), st)
+            chosen = res.candidates()[res.chosen]
         info = plan.info()
         n = max(3, args.sweep_steps)
         us = {}
-        for name, mode, out in (("fused", t3.MODE_FUSED, Y), ("sequential", t3.MODE_SEQUENTIAL, Y2),
+        for name, mode, out in (("fused", info.mode, Y), ("sequential", t3.MODE_SEQUENTIAL, Y2),
                                 ("gemm_only", t3.MODE_GEMM_ONLY, Y2), ("reduce_only", t3.MODE_REDUCE_ONLY, Y2)):
             us[name] = 1e3 * med(_time_mode(torch, plan, mode, X, W, out, st, n, 3, flush))
         same = bool(torch.equal(Y.view(torch.int16), Y2.view(torch.int16)))
@@ -434,7 +548,11 @@ def run_sweep(args):
             "tile": [info.tile_m, info.tile_n], "ring_slots": info.ring_slots, "group_tiles": info.group_tiles,
             "cluster_ctas": info.cluster_ctas, "reduce_rows": info.reduce_rows,
             "partials": "bf16" if info.partial_dtype == t3.PARTIAL_BF16 else "f32",
+            "reduce": "in place" if info.reduce == t3.REDUCE_INPLACE else "ring order",
+            "workspace_MB": round(info.workspace_bytes / 1e6, 1),
         }
+        if chosen is not None:
+            line["tuned"] = chosen
         print(json.dumps(line), flush=True)
         del X, W, Y, Y2
         torch.cuda.empty_cache()
@@ -456,8 +574,11 @@ def main():
     ap.add_argument("--sweep", action="store_true", help="configuration 5: one JSON line per shape, then exit")
     ap.add_argument("--sweep-steps", type=int, default=10)
     ap.add_argument("--sweep-filter", default="")
-    for k in ("tile_n", "group_tiles", "reducer_ctas", "reducer_warps", "reduce_rows", "stages", "ring_slots", "cluster_ctas",
-              "partial_dtype", "order"):
+    ap.add_argument("--rounds", type=int, default=5, help="interleaved companion timing: rounds")
+    ap.add_argument("--per-round", type=int, default=10, help="interleaved companion timing: flushed calls per mode and round")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the per_config block (the other configurations)")
+    ap.add_argument("--tune", action="store_true", help="let t3_plan_tune choose the configuration before timing")
+    for k in CHUNK_ARGS:
         ap.add_argument("--" + k.replace("_", "-"), dest=k, type=int, default=None)
     args = ap.parse_args()
     if args.warmup < 3 and args.impl == "ours":

@@ -33,7 +33,7 @@
 extern "C" {
 #endif
 
-#define T3_VERSION 100
+#define T3_VERSION 110
 
 typedef struct t3_plan_s *t3_plan_t;
 
@@ -89,6 +89,25 @@ typedef enum {
     T3_ORDER_STAGGERED = 1
 } t3_order_t;
 
+/* Where the R partial tiles of a region are summed (Section 4.3).
+ * T3_REDUCE_RING (default): every slice stores its own fp32 (or bf16) partial tile; once the tracker
+ * fires, reducers add the R copies in the chunk's ring order.  Deterministic, 4*R*M*N bytes of
+ * partial tiles written and read.
+ * T3_REDUCE_INPLACE: the software analog of the paper's near-memory "op-and-store" (Section 4.3; Section
+ * 7.4 suggests system-wide atomics on uncached data for hardware without it): every producer tile is
+ * ADDED into one fp32 accumulator tile per region by reductions performed at the L2
+ * (red.global.add.v4.f32); the tracker then only gates the final pass, which reads the accumulator,
+ * rounds once, writes Y and clears the accumulator for the next call.  The workspace shrinks from
+ * 4*R*M*N to 4*M*N bytes and the R-way read disappears, but the order in which the R (x split_k)
+ * contributions are added is whatever order the tiles finish in: results are NOT bit-reproducible from
+ * run to run (they stay within the tolerances; integer-valued inputs stay exact).  Needs fp32 partials
+ * and the grouped order.  After a device-side timeout call t3_plan_status before the next call: it
+ * clears the half-accumulated tiles. */
+typedef enum {
+    T3_REDUCE_RING = 0,
+    T3_REDUCE_INPLACE = 1
+} t3_reduce_t;
+
 /* debug_flags (host-made fault injection for the bounded-wait tests) */
 #define T3_DEBUG_INFLATE_EXPECTED 1   /* tracker thresholds +1: the trigger never fires, reducers time out */
 
@@ -119,7 +138,14 @@ typedef struct {
     int32_t partial_dtype;   /* t3_partial_t: storage type of the partial tiles (the "wire" type)     */
     int32_t w_layout;        /* t3_w_layout_t: how W is stored                                        */
     int32_t order;           /* t3_order_t: the producer schedule                                     */
-    int32_t reserved[1];     /* must be zero                                                         */
+    int32_t reduce;          /* t3_reduce_t: ring-order sum of stored copies, or update in place      */
+    int32_t split_k;         /* producers per (tile, slice): each takes 1/split_k of the slice's      */
+                             /* k-blocks and the tracker threshold grows to 2*R*split_k (Section 7.7: */
+                             /* split-K producers update an element more than once).  Needs            */
+                             /* reduce = T3_REDUCE_INPLACE when > 1; 0 = 1; at most 16 and at most    */
+                             /* the slice's k-blocks.  For shapes with too few tiles to fill the GPU  */
+                             /* (small M: the token-generation phase, Section 7.3).                  */
+    int32_t reserved[3];     /* must be zero                                                         */
 } t3_chunking_t;
 
 /* Geometry and cost model of a plan (all host-computed). */
@@ -143,6 +169,10 @@ typedef struct {
     int32_t partial_dtype;     /* t3_partial_t                                                */
     int32_t w_layout;          /* t3_w_layout_t                                               */
     int32_t order;             /* t3_order_t                                                  */
+    int32_t reduce;            /* t3_reduce_t                                                 */
+    int32_t split_k;           /* producers per (tile, slice), as resolved                    */
+    int32_t tuned;             /* 1 after t3_plan_tune changed or confirmed the configuration */
+    int32_t reserved0;
     int64_t workspace_bytes;   /* partial tiles (>= s_p*R*M*N) + ring + counters + control    */
     double flops;              /* 2*M*N*K                                                     */
     double bytes_gemm;         /* 2MK + 2KN + s_p*RMN : operands read once, partials written (s_p = 4 or 2) */
@@ -188,19 +218,56 @@ t3_plan_t t3_plan(int64_t M, int64_t N, int64_t K, int32_t R, t3_dtype_t dtype,
  * of the R partial products added in fp32 in the ring order
  * (c-1, c-2, ..., c) mod R (Section 4.1's four-device example).  The result is
  * bit-identical from run to run and between FUSED and SEQUENTIAL modes.
- * One call in flight per plan, and one t3 kernel in flight per device: the
- * kernel is persistent (one CTA per SM, all CTA pairs must be resident
- * together because reducers wait on tiles other pairs produce), so two calls
- * overlapping on one GPU from different streams can starve each other until
- * the bounded waits run out (T3_ERR_TIMEOUT), never hang.  Serialise calls
- * per device.  Host-detectable errors return a negative code and enqueue
- * nothing; device-side timeouts are reported by t3_plan_status.
+ * One call in flight per plan.  The kernel is persistent (one CTA per SM, all
+ * CTA pairs must be resident together because reducers wait on tiles other
+ * pairs produce), so two t3 kernels must never share a GPU.  The library
+ * sees to that itself: every launch made through a plan first waits, on its
+ * stream, for an event recorded after the previous t3 launch on the same
+ * device (whatever plan or stream that was), without blocking the host;
+ * calls from several streams or host threads therefore run one after the
+ * other on the GPU.  (Not inside a stream capture: a captured call is ordered
+ * by its graph alone.  Not for t3_gemm_rs_static, which creates nothing.)
+ * The plan must be used with the device it was made on current
+ * (T3_ERR_DEVICE otherwise).  Host-detectable errors return a negative code
+ * and enqueue nothing; device-side timeouts are reported by t3_plan_status;
+ * a timeout left uncollected does not disturb later calls on the plan.
  * In FUSED mode a call enqueues exactly one kernel and nothing else (the
  * kernel re-arms the tracker itself), so calls can be recorded into a CUDA
  * graph by stream capture after one ordinary call per plan and (X, W) pair
  * (the first call with new operand pointers encodes their tensor maps).
  */
 int t3_gemm_rs(t3_plan_t plan, const void *X, const void *W, void *Y, void *stream);
+
+/*
+ * t3_gemm_rs_ex - t3_gemm_rs with element-wise work fused on the reduced chunk
+ * (Section 7.6: the operators that follow the all-reduce - bias, dropout,
+ * residual add - can run on the reduce-scattered sub-array, before the
+ * all-gather, so each device does 1/R of that work and Y is written once).
+ * Per element, in fp32, each step rounded to nearest even and never fused:
+ *     y = ((sum_r P_r + bias[n]) * (keep[m][n] ? keep_scale : 0)) + residual[m][n]
+ * followed by the single rounding to Y's type.  Steps whose pointer is NULL
+ * are skipped; epi == NULL is t3_gemm_rs.  All pointers are device pointers,
+ * 16-byte aligned, caller-owned, read only:
+ *   bias      [N]    bf16 or fp32 (bias_dtype)
+ *   residual  [M,N]  row-major, bf16 or fp32 (residual_dtype); may not alias Y
+ *   keep      [M,N]  bytes, non-zero = keep: a dropout mask the CALLER drew
+ *                    (the library draws no random numbers); keep_scale is
+ *                    the caller's 1/(1-p)
+ * Works in every mode that writes Y (the sequential baseline's reduce kernel
+ * applies the same tail, so FUSED and SEQUENTIAL stay bit-identical).
+ */
+typedef enum { T3_EPI_BF16 = 0, T3_EPI_F32 = 1 } t3_epi_dtype_t;
+typedef struct {
+    const void *bias;
+    const void *residual;
+    const void *keep;
+    float keep_scale;
+    int32_t bias_dtype;        /* t3_epi_dtype_t */
+    int32_t residual_dtype;    /* t3_epi_dtype_t */
+    int32_t reserved;          /* must be zero   */
+} t3_epilogue_t;
+int t3_gemm_rs_ex(t3_plan_t plan, const void *X, const void *W, void *Y,
+                  const t3_epilogue_t *epi /* host or NULL */, void *stream);
 
 /* Same, in an explicit mode (the bench times FUSED, SEQUENTIAL, GEMM_ONLY and
  * REDUCE_ONLY on one plan so that all share one workspace and tile shape;
@@ -265,6 +332,32 @@ int t3_gemm_rs_host(t3_plan_t plan, const void *X_host, const void *W_host, void
 int t3_gemm_rs_static(int64_t M, int64_t N, int64_t K, int32_t R, t3_dtype_t dtype, const void *X,
                       const void *W, void *Y, void *stream);
 
+/*
+ * t3_plan_tune - choose the plan's configuration by measurement (the analog of
+ * Section 4.5: the paper's memory-controller arbitration learns its threshold
+ * from the producer kernel's behaviour while it runs alone in the first
+ * stage; here a short trial on the real operands decides how the reduction
+ * shares the GPU with the GEMM).  Runs the op a few times per candidate on
+ * `stream`, timing with CUDA events, and keeps the fastest of
+ *   { fused with the L2 ring, fused with full partial buffers, sequential }
+ *   x reduce_rows { 16, 32 } x cluster_ctas { 2, 4 where available } x group height { g, g/2 }
+ * that fit the plan's existing workspace (nothing is allocated).  A candidate
+ * replaces the current configuration only if it is at least 2 % faster.  All
+ * candidates produce the same bits, so tuning never changes a result
+ * (T3_REDUCE_INPLACE plans: within its stated non-determinism).
+ * Synchronous: returns after the trials; Y holds a valid result.  out (host,
+ * may be NULL) receives what was tried.  Call it once, before steady-state
+ * use and outside stream capture.
+ */
+typedef struct {
+    int32_t n_tried;
+    int32_t chosen;              /* index into the arrays below                                   */
+    int32_t mode[48], ring_slots[48], reduce_rows[48], cluster_ctas[48], group_tiles[48];
+    float us[48];                /* median microseconds per call of each candidate                */
+} t3_tune_t;
+int t3_plan_tune(t3_plan_t plan, const void *X, const void *W, void *Y, void *stream,
+                 t3_tune_t *out /* host or NULL */);
+
 /* t3_destroy - synchronises the device, frees the workspace. NULL is a no-op. */
 int t3_destroy(t3_plan_t plan);
 
@@ -289,11 +382,40 @@ int t3_plan_status(t3_plan_t plan, t3_status_t *out /* host */);
 int t3_plan_partials(t3_plan_t plan, void **partials /* host, receives device ptr */,
                      int64_t *bytes /* host or NULL */);
 
+/* Device pointer to, and size of, the recycled ring of region slots that the
+ * FUSED mode writes its partial tiles to (NULL and 0 when the plan has no
+ * ring and FUSED uses the full buffers).  Contents opaque; a test may poison
+ * it between calls. */
+int t3_plan_ring(t3_plan_t plan, void **ring /* host, receives device ptr */,
+                 int64_t *bytes /* host or NULL */);
+
+/*
+ * t3_plan_timeline - where the time of the plan's last FUSED call went
+ * (Section 5.1.3 compares against an ideal overlap; this splits the fused
+ * kernel's own time the same way).  Every CTA records the GPU's global
+ * nanosecond timer at four points; the call synchronises the plan's last
+ * stream and reduces them:
+ *   total_us    first CTA start -> last CTA end
+ *   produce_us  first CTA start -> last tracker update (the last partial tile
+ *               of the GEMM has landed: the producer phase, run under the
+ *               reduction's contention)
+ *   tail_us     last tracker update -> last reduced item (reduction that
+ *               nothing can overlap with any more)
+ *   drain_us    last reduced item -> last CTA end (teardown)
+ */
+typedef struct {
+    double total_us, produce_us, tail_us, drain_us;
+    int32_t ctas;
+    int32_t reserved;
+} t3_timeline_t;
+int t3_plan_timeline(t3_plan_t plan, t3_timeline_t *out /* host */);
+
 /* Writes the partial products held in the full partial buffers (as left by
  * the last SEQUENTIAL or GEMM_ONLY call) to dst as plain row-major fp32
  * [R][M][N] (device pointer, caller-owned, 4*R*M*N bytes), asynchronously on
  * `stream`.  Lets a test check the producer GEMM and the reduction stage
- * (Section 2.3's element-wise sum) separately. */
+ * (Section 2.3's element-wise sum) separately.  T3_ERR_UNSUPPORTED for
+ * T3_REDUCE_INPLACE plans (no per-slice copies exist). */
 int t3_plan_export_partials(t3_plan_t plan, void *dst /* device */, void *stream);
 
 /* Host-only (no GPU needed): the geometry t3_plan would choose. */

@@ -56,6 +56,19 @@ constexpr int RED_WARPS_GEMM_CTA = 8;               // reducer warps inside a CT
 enum Where { W_TMA = 1, W_MMA = 2, W_EPI = 3, W_RED = 4, W_PUB = 5 };
 constexpr int ERR_TIMEOUT = -6;         // = T3_ERR_TIMEOUT
 
+// Element-wise operators applied to the reduced sum before its single rounding (Section 7.6: the work
+// that follows the all-reduce - bias, dropout, residual add - done on the reduce-scattered chunk):
+//   y = ((sum + bias[n]) * (keep[m][n] ? keep_scale : 0)) + residual[m][n]
+// each step one fp32 operation, rounded to nearest even, never contracted.  A NULL pointer skips its step.
+struct EpiOps {
+    const void* bias;           // [N] bf16 or fp32
+    const void* residual;       // [M][N] bf16 or fp32
+    const uint8_t* keep;        // [M][N] bytes, non-zero = keep (a dropout mask drawn by the caller)
+    float keep_scale;           // 1 / (1 - p)
+    int bias_f32, residual_f32;
+    int any;                    // 0: nothing to do (plain reduce-scatter)
+};
+
 struct alignas(64) KParams {
     CUtensorMap tmX;        // bf16 X viewed as (K_r, R, M)
     CUtensorMap tmW;        // bf16 W[N][K] viewed as (K_r, R, N); or, with w_kn, W[K][N] viewed as (N, K_r, R)
@@ -86,17 +99,15 @@ struct alignas(64) KParams {
     int out_f32;
     uint32_t expected;      // tracker threshold per region
     unsigned long long timeout_ns;
+    uint32_t epoch;         // launch number of the owning plan (> 0): ctl[2] == epoch means "this launch is aborting"
+    int split_k;            // producers per (tile, slice): schedule slice index rv = r * split_k + part (in-place mode only when > 1)
+    int inplace;            // 1: update-in-place reduction (Section 4.3's analog): the epilogues add every slice's
+                            // tile into ONE fp32 accumulator tile per region with L2 reductions; the tracker then
+                            // gates only the final convert / store pass, which also clears the accumulator
+    EpiOps epi;             // element-wise work fused on the reduced chunk (Section 7.6)
+    unsigned long long* trace;   // [grid][4] globaltimer: start, last tracker update, last reduced item, end; or NULL
 };
 
-#ifdef T3_PROFILE
-// debug build only: per-CTA cycle counts of where the single-thread roles spend their time
-__device__ long long g_prof[160 * 16];
-#define PROF_T0(var) long long var = clock64()
-#define PROF_ADD(acc, var) acc += clock64() - var
-#else
-#define PROF_T0(var)
-#define PROF_ADD(acc, var)
-#endif
 
 // k-blocks of slice r.  Slice r starts r * K_r elements into a row; when K_r is not a multiple of 64
 // that is not on a 128-byte line for every r, and a 64-wide box would straddle two lines in each row.
@@ -109,17 +120,41 @@ __device__ __forceinline__ int slice_k_shift(const KParams& p, int r) {
 __device__ __forceinline__ int slice_k_blocks(const KParams& p, int shift) {
     return (p.Kr + shift + BK - 1) / BK;
 }
+// A producer job's share of its slice: the schedule's slice index rv names slice r = rv / split_k and
+// part rv % split_k of that slice's nkb k-blocks, [kb0, kb1).
+__device__ __forceinline__ void job_k_range(const KParams& p, int rv, int& r, int& shift, int& nkb, int& kb0, int& kb1) {
+    r = rv;
+    shift = slice_k_shift(p, r);
+    nkb = slice_k_blocks(p, shift);
+    kb0 = 0;
+    kb1 = nkb;
+    if (p.split_k > 1) {
+        r = rv / p.split_k;
+        const int part = rv - r * p.split_k;
+        shift = slice_k_shift(p, r);
+        nkb = slice_k_blocks(p, shift);
+        kb0 = part * nkb / p.split_k;
+        kb1 = (part + 1) * nkb / p.split_k;
+    }
+}
 
 // ---------------------------------------------------------------------------
 // bounded waits
 // ---------------------------------------------------------------------------
+// Records the first failure in the status words (kept until the host collects them) and marks THIS launch
+// as aborting (ctl[2] = epoch), which is what the other CTAs' waits look at: a status left uncollected by
+// an earlier launch does not disturb later ones.
 __device__ __forceinline__ void report(const KParams& p, int where, int detail) {
     if (atomicCAS(reinterpret_cast<int*>(p.status), 0, ERR_TIMEOUT) == 0) {
         p.status[1] = where;
         p.status[2] = static_cast<int>(blockIdx.x);
         p.status[3] = detail;
-        __threadfence();
     }
+    atomicExch(&p.ctl[2], p.epoch);
+    __threadfence();
+}
+__device__ __forceinline__ bool launch_aborting(const KParams& p) {
+    return *reinterpret_cast<volatile uint32_t*>(&p.ctl[2]) == p.epoch;
 }
 
 // Returns false when the wait ran out (or the CTA is already aborting).
@@ -165,7 +200,7 @@ __device__ __forceinline__ bool wait_region(const KParams& p, const uint32_t* cn
         if (static_cast<int32_t>(ld_acquire_gpu(cnt) - p.expected) >= 0) return true;
         __nanosleep(200);
         if ((++polls & 63) == 0) {
-            if (*reinterpret_cast<volatile int32_t*>(p.status) != 0) return false;
+            if (launch_aborting(p)) return false;
             if (globaltimer_ns() - t0 > p.timeout_ns) {
                 report(p, W_RED, region);
                 return false;
@@ -178,20 +213,69 @@ __device__ __forceinline__ bool wait_region(const KParams& p, const uint32_t* cn
 // the reduction (Section 2.3's element-wise sum): per element, sequential fp32 adds of the R
 // partials in the chunk's ring order.
 // ---------------------------------------------------------------------------
-// One row's eight neighbouring outputs (columns col .. col + 7), rounded once to the output type.
-__device__ __forceinline__ void store_y_8(void* Y, int N, int row, int col, const float2 (&a)[4], int out_f32) {
+// eight neighbouring values of a bf16 or fp32 array, as floats
+__device__ __forceinline__ void load_8(const void* base, size_t idx, int is_f32, float (&v)[8]) {
+    if (is_f32) {
+        const float4* src = reinterpret_cast<const float4*>(static_cast<const float*>(base) + idx);
+        const float4 lo = src[0], hi = src[1];
+        v[0] = lo.x; v[1] = lo.y; v[2] = lo.z; v[3] = lo.w; v[4] = hi.x; v[5] = hi.y; v[6] = hi.z; v[7] = hi.w;
+    } else {
+        const uint4 u = *reinterpret_cast<const uint4*>(static_cast<const __nv_bfloat16*>(base) + idx);
+        const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            v[2 * k] = __uint_as_float(w[k] << 16);
+            v[2 * k + 1] = __uint_as_float(w[k] & 0xffff0000u);
+        }
+    }
+}
+
+// The element-wise tail of Section 7.6 on one row's eight neighbouring sums (columns col .. col + 7).  A real
+// call, not inlined: its registers are then needed only while it runs, not across the reducers' load rounds.
+__device__ __noinline__ void apply_epi_8(const EpiOps& eo, int N, int row, int col, float (&v)[8]) {
     const size_t off = static_cast<size_t>(row) * static_cast<size_t>(N) + col;
+    // issue the per-element loads first, then the (cached) bias
+    uint2 km = make_uint2(0x01010101u, 0x01010101u);
+    float res[8];
+    if (eo.keep) km = *reinterpret_cast<const uint2*>(eo.keep + off);
+    if (eo.residual) load_8(eo.residual, off, eo.residual_f32, res);
+    if (eo.bias) {
+        float b[8];
+        load_8(eo.bias, static_cast<size_t>(col), eo.bias_f32, b);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = __fadd_rn(v[i], b[i]);
+    }
+    if (eo.keep) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+            const uint32_t byte = ((i < 4 ? km.x : km.y) >> (8 * (i & 3))) & 0xffu;
+            v[i] = __fmul_rn(v[i], byte ? eo.keep_scale : 0.0f);
+        }
+    }
+    if (eo.residual) {
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v[i] = __fadd_rn(v[i], res[i]);
+    }
+}
+
+// One row's eight neighbouring outputs (columns col .. col + 7): the element-wise tail, if any, then one
+// rounding to the output type.
+__device__ __forceinline__ void store_y_8(void* Y, int N, int row, int col, const float2 (&a)[4], int out_f32,
+                                          const EpiOps& eo) {
+    const size_t off = static_cast<size_t>(row) * static_cast<size_t>(N) + col;
+    float v[8] = {a[0].x, a[0].y, a[1].x, a[1].y, a[2].x, a[2].y, a[3].x, a[3].y};
+    if (eo.any) apply_epi_8(eo, N, row, col, v);
     if (out_f32) {
         float4* dst = reinterpret_cast<float4*>(static_cast<float*>(Y) + off);
-        dst[0] = make_float4(a[0].x, a[0].y, a[1].x, a[1].y);
-        dst[1] = make_float4(a[2].x, a[2].y, a[3].x, a[3].y);
+        dst[0] = make_float4(v[0], v[1], v[2], v[3]);
+        dst[1] = make_float4(v[4], v[5], v[6], v[7]);
     } else {
         uint4 u;
         __nv_bfloat162 h;
-        h = __floats2bfloat162_rn(a[0].x, a[0].y); u.x = *reinterpret_cast<uint32_t*>(&h);
-        h = __floats2bfloat162_rn(a[1].x, a[1].y); u.y = *reinterpret_cast<uint32_t*>(&h);
-        h = __floats2bfloat162_rn(a[2].x, a[2].y); u.z = *reinterpret_cast<uint32_t*>(&h);
-        h = __floats2bfloat162_rn(a[3].x, a[3].y); u.w = *reinterpret_cast<uint32_t*>(&h);
+        h = __floats2bfloat162_rn(v[0], v[1]); u.x = *reinterpret_cast<uint32_t*>(&h);
+        h = __floats2bfloat162_rn(v[2], v[3]); u.y = *reinterpret_cast<uint32_t*>(&h);
+        h = __floats2bfloat162_rn(v[4], v[5]); u.z = *reinterpret_cast<uint32_t*>(&h);
+        h = __floats2bfloat162_rn(v[6], v[7]); u.w = *reinterpret_cast<uint32_t*>(&h);
         *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(Y) + off) = u;
     }
 }
@@ -217,7 +301,8 @@ __device__ __forceinline__ void quad_exchange(float2& lo, float2& hi, int q) {
 template <int B>
 __device__ __forceinline__ void reduce_row_group(const float* __restrict__ chunk, size_t slice_stride, int rowsel,
                                                  void* Y, int M, int N, int R, int chunk_rows, int out_f32,
-                                                 int row_base, int col_base, int ncols_left, int lane) {
+                                                 int row_base, int col_base, int ncols_left, int lane,
+                                                 const EpiOps& eo) {
     const int g = lane >> 2, q = lane & 3;
     // float4 index of (rowsel, jp, lane): ((2 * rowsel + jp) * 32 + lane)
     const float* pos = chunk + (static_cast<size_t>(2 * rowsel) * 32 + lane) * 4;
@@ -256,7 +341,7 @@ __device__ __forceinline__ void reduce_row_group(const float* __restrict__ chunk
     quad_exchange<1>(a[2], a[3], q);
     quad_exchange<2>(a[0], a[2], q);
     quad_exchange<2>(a[1], a[3], q);
-    if (row < M && 8 * q < ncols_left) store_y_8(Y, N, row, col_base + 8 * q, a, out_f32);
+    if (row < M && 8 * q < ncols_left) store_y_8(Y, N, row, col_base + 8 * q, a, out_f32, eo);
 }
 
 // 16-bit partial tiles: the same reduction of one 8-row group; a lane reads its row's eight values of a
@@ -265,7 +350,8 @@ __device__ __forceinline__ void reduce_row_group(const float* __restrict__ chunk
 template <int B>
 __device__ __forceinline__ void reduce_row_group_bf16(const __nv_bfloat16* __restrict__ chunk, size_t slice_stride,
                                                       int rowsel, void* Y, int M, int N, int R, int chunk_rows,
-                                                      int out_f32, int row_base, int col_base, int ncols_left, int lane) {
+                                                      int out_f32, int row_base, int col_base, int ncols_left, int lane,
+                                                      const EpiOps& eo) {
     const int g = lane >> 2, q = lane & 3;
     const __nv_bfloat16* pos = chunk + (static_cast<size_t>(rowsel) * 32 + lane) * 8;
     const int row = row_base + 8 * rowsel + g;
@@ -300,27 +386,64 @@ __device__ __forceinline__ void reduce_row_group_bf16(const __nv_bfloat16* __res
     quad_exchange<1>(a[2], a[3], q);
     quad_exchange<2>(a[0], a[2], q);
     quad_exchange<2>(a[1], a[3], q);
-    if (row < M && 8 * q < ncols_left) store_y_8(Y, N, row, col_base + 8 * q, a, out_f32);
+    if (row < M && 8 * q < ncols_left) store_y_8(Y, N, row, col_base + 8 * q, a, out_f32, eo);
+}
+
+// Update-in-place mode: the chunk holds the finished sums.  All row groups [first, end) of the item (at
+// most four) are read with their loads in flight together, cleared for the next call, regrouped among
+// the four lanes of a row and written to Y.
+__device__ __noinline__ void finish_item_inplace(const float* __restrict__ chunk, int first, int end, void* Y, int M, int N,
+                                                    int out_f32, int row_base, int col_base, int ncols_left, int lane,
+                                                    const EpiOps& eo) {
+    const int g = lane >> 2, q = lane & 3;
+    float* pos = const_cast<float*>(chunk) + lane * 4;
+    float4 x[4][2];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        if (first + i < end) {
+            x[i][0] = ld_partial_v4(pos + static_cast<size_t>(2 * (first + i)) * 128);
+            x[i][1] = ld_partial_v4(pos + static_cast<size_t>(2 * (first + i) + 1) * 128);
+        }
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+        if (first + i < end) {
+            float* z = pos + static_cast<size_t>(2 * (first + i)) * 128;
+            *reinterpret_cast<float4*>(z) = make_float4(0.f, 0.f, 0.f, 0.f);
+            *reinterpret_cast<float4*>(z + 128) = make_float4(0.f, 0.f, 0.f, 0.f);
+            float2 a[4] = {make_float2(x[i][0].x, x[i][0].y), make_float2(x[i][0].z, x[i][0].w),
+                           make_float2(x[i][1].x, x[i][1].y), make_float2(x[i][1].z, x[i][1].w)};
+            quad_exchange<1>(a[0], a[1], q);
+            quad_exchange<1>(a[2], a[3], q);
+            quad_exchange<2>(a[0], a[2], q);
+            quad_exchange<2>(a[1], a[3], q);
+            const int row = row_base + 8 * (first + i) + g;
+            if (row < M && 8 * q < ncols_left) store_y_8(Y, N, row, col_base + 8 * q, a, out_f32, eo);
+        }
 }
 
 // One reducer item: `rows` (8, 16 or 32) rows of the chunk starting at block row `row_in_block`.
 // chunk: the chunk's storage in slice 0 (fp32, or bf16 when partial_bf16); slice_stride in elements.
+// inplace: the chunk is the region's single fp32 accumulator (already the sum of all slices): read, clear, write Y.
 __device__ __forceinline__ void reduce_item(const void* __restrict__ chunk, size_t slice_stride, int partial_bf16,
                                             int row_in_block, int rows, void* Y, int M, int N, int R, int chunk_rows,
-                                            int out_f32, int row_base, int col_base, int ncols_left, int lane) {
+                                            int out_f32, int row_base, int col_base, int ncols_left, int lane,
+                                            const EpiOps& eo, int inplace) {
     const int first = row_in_block >> 3;
     int end = (row_in_block + rows) >> 3;
     if (row_base + 8 * end > M) end = (M - row_base + 7) >> 3;     // the rest of the block is padding
-    if (partial_bf16) {
+    if (inplace) {
+        finish_item_inplace(static_cast<const float*>(chunk), first, end, Y, M, N, out_f32, row_base, col_base, ncols_left,
+                            lane, eo);
+    } else if (partial_bf16) {
 #pragma unroll 1
         for (int rowsel = first; rowsel < end; ++rowsel)
             reduce_row_group_bf16<8>(static_cast<const __nv_bfloat16*>(chunk), slice_stride, rowsel, Y, M, N, R, chunk_rows,
-                                      out_f32, row_base, col_base, ncols_left, lane);
+                                      out_f32, row_base, col_base, ncols_left, lane, eo);
     } else {
 #pragma unroll 1
         for (int rowsel = first; rowsel < end; ++rowsel)
             reduce_row_group<8>(static_cast<const float*>(chunk), slice_stride, rowsel, Y, M, N, R, chunk_rows, out_f32,
-                                row_base, col_base, ncols_left, lane);
+                                row_base, col_base, ncols_left, lane, eo);
     }
 }
 
@@ -336,6 +459,23 @@ __device__ __forceinline__ void epi_store_frag(const uint32_t (&lo)[16], const u
         const uint32_t* src = rowsel < 2 ? lo : hi;
         asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p0 + i * 128), "r"(src[8 * jp + 2 * half]),
                      "r"(src[8 * jp + 2 * half + 1]), "r"(src[8 * jp + 4 + 2 * half]), "r"(src[8 * jp + 4 + 2 * half + 1])
+                     : "memory");
+    }
+}
+
+// Update-in-place variant (Section 4.3's near-memory "op-and-store", done here by the L2's reduction
+// units): the same eight 128-bit accesses per lane, each adding its four floats into the region's
+// accumulator tile instead of storing them into the slice's own copy.
+__device__ __forceinline__ void epi_red_frag(const uint32_t (&lo)[16], const uint32_t (&hi)[16], int lane,
+                                             float* __restrict__ chunk) {
+    float* p0 = chunk + lane * 4;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int rowsel = i >> 1, jp = i & 1, half = rowsel & 1;
+        const uint32_t* src = rowsel < 2 ? lo : hi;
+        asm volatile("red.relaxed.gpu.global.add.v4.f32 [%0], {%1, %2, %3, %4};" ::"l"(p0 + i * 128),
+                     "f"(__uint_as_float(src[8 * jp + 2 * half])), "f"(__uint_as_float(src[8 * jp + 2 * half + 1])),
+                     "f"(__uint_as_float(src[8 * jp + 4 + 2 * half])), "f"(__uint_as_float(src[8 * jp + 4 + 2 * half + 1]))
                      : "memory");
     }
 }
@@ -377,6 +517,7 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
     __shared__ uint32_t tmem_holder;
     __shared__ int abort_flag_s;
     __shared__ int is_last_s;
+    __shared__ unsigned long long trace_s[3];                 // kernel start, last tracker update, last reduced item
     volatile int* abort_flag = &abort_flag_s;
 
     const int warp = __shfl_sync(0xffffffffu, static_cast<int>(threadIdx.x) >> 5, 0);
@@ -393,6 +534,9 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
     if (threadIdx.x == 0) {
         abort_flag_s = 0;
         is_last_s = 0;
+        trace_s[0] = globaltimer_ns();
+        trace_s[1] = 0ull;
+        trace_s[2] = 0ull;
         for (int s = 0; s < p.stages; ++s) {
             mbar_init(smem_u32(&bar_full[s]), 1);
             mbar_init(smem_u32(&bar_empty[s]), CLUSTER / CTA_PAIR);
@@ -427,27 +571,21 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
             int s = 0;
             uint32_t ph = 0;
             bool ok = true;
-#ifdef T3_PROFILE
-            long long prof_wait = 0; const long long prof_start = clock64();
-#endif
             const uint32_t full0 = mapa_cluster(smem_u32(&bar_full[0]), lead);   // the pair leader's full barriers
             const int a_row_off = static_cast<int>(half) * BM;
             const int b_row_off = static_cast<int>(half) * (p.BN >> 1);
 #pragma unroll 1
             for (int j = pair; ok && j < p.sched.n_jobs; j += gemm_pairs) {
-                int mt, nt, r;
-                decode_job(p.sched, j, mt, nt, r);
+                int mt, nt, rv, r, shift, nkb, kb0, kb1;
+                decode_job(p.sched, j, mt, nt, rv);
+                job_k_range(p, rv, r, shift, nkb, kb0, kb1);
                 const int a_row = mt * BMJ + a_row_off, b_row = nt * p.BN + b_row_off;
-                const int shift = slice_k_shift(p, r);
-                const int nkb = slice_k_blocks(p, shift);
 #pragma unroll 1
-                for (int kb = 0; kb < nkb; ++kb) {
-                    PROF_T0(tw);
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!mbar_wait(p, smem_u32(&bar_empty[s]), ph ^ 1u, abort_flag, W_TMA, j)) {
                         ok = false;
                         break;
                     }
-                    PROF_ADD(prof_wait, tw);
                     // stage layout: [A k-block][half B k-block]
                     const uint32_t dst = tiles + static_cast<uint32_t>(s) * p.stage_bytes;
                     const uint32_t dstB = dst + p.a_bytes;
@@ -485,9 +623,6 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
             }
-#ifdef T3_PROFILE
-            if (lane == 0) { g_prof[blockIdx.x * 16 + 0] = prof_wait; g_prof[blockIdx.x * 16 + 1] = clock64() - prof_start; }
-#endif
         }
         __syncwarp();
       } else if (is_gemm && warp == MMA_WARP) {
@@ -506,31 +641,22 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
             int s = 0, jl = 0, acc = 0;
             uint32_t ph = 0, soff = 0, acc_ph = 0;
             bool ok = true;
-#ifdef T3_PROFILE
-            long long prof_wfull = 0, prof_wtempty = 0, prof_issue = 0; const long long prof_start = clock64();
-#endif
 #pragma unroll 1
             for (int j = pair; ok && j < p.sched.n_jobs; j += gemm_pairs, ++jl) {
-                int mt, nt, r;
-                decode_job(p.sched, j, mt, nt, r);
-                const int shift = slice_k_shift(p, r);
-                const int nkb = slice_k_blocks(p, shift);
+                int mt, nt, rv, r, shift, nkb, kb0, kb1;
+                decode_job(p.sched, j, mt, nt, rv);
+                job_k_range(p, rv, r, shift, nkb, kb0, kb1);
                 const int first_step = shift / UMMA_K;                                   // leading all-zero k-steps of block 0
                 const int last_steps = (p.Kr + shift - (nkb - 1) * BK + UMMA_K - 1) / UMMA_K;   // k-steps with data in the last block
-                PROF_T0(te);
                 if (!mbar_wait<true>(p, smem_u32(&bar_tempty[acc]), acc_ph ^ 1u, abort_flag, W_MMA, j)) break;
-                PROF_ADD(prof_wtempty, te);
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(acc * p.acc_stride);
 #pragma unroll 1
-                for (int kb = 0; kb < nkb; ++kb) {
-                    PROF_T0(tf);
+                for (int kb = kb0; kb < kb1; ++kb) {
                     if (!mbar_wait(p, smem_u32(&bar_full[s]), ph, abort_flag, W_MMA, j)) {
                         ok = false;
                         break;
                     }
-                    PROF_ADD(prof_wfull, tf);
-                    PROF_T0(ti);
                     tc_fence_after();
                     const uint64_t a_desc = a_desc0 + soff, b_desc = b_desc0 + soff;
                     const int ka = kb == 0 ? first_step : 0;
@@ -538,7 +664,7 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                     if (elect_one_sync()) {
                         // +32 bytes along K inside the 128-byte swizzle row = +2 in the address field
                         if (ka == 0 && kz == BK / UMMA_K) {
-                            umma_bf16_ss_pair(d_tmem, a_desc, b_desc, idesc, static_cast<uint32_t>(kb != 0));
+                            umma_bf16_ss_pair(d_tmem, a_desc, b_desc, idesc, static_cast<uint32_t>(kb != kb0));
                             umma_bf16_ss_pair(d_tmem, a_desc + 2, b_desc + b_step, idesc, 1u);
                             umma_bf16_ss_pair(d_tmem, a_desc + 4, b_desc + 2 * b_step, idesc, 1u);
                             umma_bf16_ss_pair(d_tmem, a_desc + 6, b_desc + 3 * b_step, idesc, 1u);
@@ -547,27 +673,19 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
 #pragma unroll 1
                             for (int k = ka; k < kz; ++k)
                                 umma_bf16_ss_pair(d_tmem, a_desc + static_cast<uint64_t>(2 * k), b_desc + static_cast<uint64_t>(k) * b_step,
-                                                  idesc, static_cast<uint32_t>(kb != 0 || k != ka));
+                                                  idesc, static_cast<uint32_t>(kb != kb0 || k != ka));
                         }
                         // the stage is reusable once these MMAs retire: tell every CTA that fetches into it
                         umma_commit_pair_mask(smem_u32(&bar_empty[s]), all_mask);
                         // accumulator complete in both CTAs of the pair
-                        if (kb == nkb - 1) umma_commit_pair_mask(smem_u32(&bar_tfull[acc]), pair_mask);
+                        if (kb == kb1 - 1) umma_commit_pair_mask(smem_u32(&bar_tfull[acc]), pair_mask);
                     }
                     __syncwarp();
-                    PROF_ADD(prof_issue, ti);
                     soff += stage_units;
                     if (++s == p.stages) { s = 0; ph ^= 1u; soff = 0; }
                 }
                 if (++acc == p.n_acc) { acc = 0; acc_ph ^= 1u; }
             }
-#ifdef T3_PROFILE
-            if (lane == 0) {
-                g_prof[blockIdx.x * 16 + 2] = prof_wfull; g_prof[blockIdx.x * 16 + 3] = prof_wtempty;
-                g_prof[blockIdx.x * 16 + 4] = prof_issue; g_prof[blockIdx.x * 16 + 5] = clock64() - prof_start;
-                g_prof[blockIdx.x * 16 + 6] = jl;
-            }
-#endif
         }
         __syncwarp();
       } else if (is_gemm && warp == PUB_WARP) {
@@ -587,6 +705,7 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                     mbar_arrive(smem_u32(&bar_taken[acc]));
                     __threadfence();                                   // gpu-scope release of the four warps' stores
                     red_relaxed_gpu_add(&p.counters[mt * p.sched.n_nt + nt], 1u);
+                    *reinterpret_cast<volatile unsigned long long*>(&trace_s[1]) = globaltimer_ns();
                 }
                 __syncwarp();
                 if (++acc == p.n_acc) { acc = 0; acc_ph ^= 1u; }
@@ -618,9 +737,6 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                 next_slot_seen = ld_acquire_gpu(next_slot_done);
             }
         }
-#ifdef T3_PROFILE
-        long long prof_wtfull = 0, prof_fence = 0; const long long prof_start = clock64();
-#endif
 #pragma unroll 1
         for (int j = pair; j < p.sched.n_jobs; j += gemm_pairs, ++jl) {
             int mt, nt, r, seq;
@@ -643,11 +759,8 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                     next_slot_seen = ld_acquire_gpu(next_slot_done);
                 }
             }
-            PROF_T0(tt);
             if (!mbar_wait(p, smem_u32(&bar_tfull[acc]), acc_ph, abort_flag, W_EPI, j)) break;
-            PROF_ADD(prof_wtfull, tt);
             tc_fence_after();
-            PROF_T0(tsl);
             if (slot_done != nullptr && slot_seen < slot_need) {
                 const uint64_t t0 = globaltimer_ns();
                 bool freed = true;
@@ -663,14 +776,13 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                 }
             }
             __syncwarp();
-            PROF_ADD(prof_fence, tsl);
             const int col0 = nt * p.BN;
             const int ncols = min(p.BN, p.N - col0);
             const int nchunks = (ncols + EPI_CHUNK - 1) / EPI_CHUNK;
             // this warp's row block (half * 4 + q) of slice r's tile in the region's slot
             const int slot = p.ring_slots > 0 ? seq % p.ring_slots : mt * p.sched.n_nt + nt;
             const size_t dst_off = static_cast<size_t>(slot) * static_cast<size_t>(p.slot_elems) +
-                                   static_cast<size_t>(r) * static_cast<size_t>(p.tile_elems) +
+                                   static_cast<size_t>(p.inplace ? 0 : r) * static_cast<size_t>(p.tile_elems) +
                                    static_cast<size_t>((static_cast<int>(half) * EPI_WARPS + q) * p.sched.nc) * FRAG_ELEMS;
             float* dst = p.partials + dst_off;
             __nv_bfloat16* dst16 = reinterpret_cast<__nv_bfloat16*>(p.partials) + dst_off;
@@ -692,7 +804,8 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster_relaxed(tempty0 + static_cast<uint32_t>(acc) * 8u);
                 }
-                if (p.partial_bf16) epi_store_frag_bf16(alo, ahi, lane, dst16 + ci * FRAG_ELEMS);
+                if (p.inplace) epi_red_frag(alo, ahi, lane, dst + ci * FRAG_ELEMS);
+                else if (p.partial_bf16) epi_store_frag_bf16(alo, ahi, lane, dst16 + ci * FRAG_ELEMS);
                 else epi_store_frag(alo, ahi, lane, dst + ci * FRAG_ELEMS);
                 if (ci + 1 < nchunks) {
                     tmem_ld_wait();
@@ -704,7 +817,8 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                         __syncwarp();
                         if (lane == 0) mbar_arrive_cluster_relaxed(tempty0 + static_cast<uint32_t>(acc) * 8u);
                     }
-                    if (p.partial_bf16) epi_store_frag_bf16(blo, bhi, lane, dst16 + (ci + 1) * FRAG_ELEMS);
+                    if (p.inplace) epi_red_frag(blo, bhi, lane, dst + (ci + 1) * FRAG_ELEMS);
+                    else if (p.partial_bf16) epi_store_frag_bf16(blo, bhi, lane, dst16 + (ci + 1) * FRAG_ELEMS);
                     else epi_store_frag(blo, bhi, lane, dst + (ci + 1) * FRAG_ELEMS);
                 }
             }
@@ -714,12 +828,6 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
             if (lane == 0) mbar_arrive(smem_u32(&bar_stored[acc]));
             if (++acc == p.n_acc) { acc = 0; acc_ph ^= 1u; }
         }
-#ifdef T3_PROFILE
-        if (lane == 0 && warp == FIRST_EPI_WARP) {
-            g_prof[blockIdx.x * 16 + 8] = prof_wtfull; g_prof[blockIdx.x * 16 + 9] = clock64() - prof_start;
-            g_prof[blockIdx.x * 16 + 14] = prof_fence;
-        }
-#endif
         __syncwarp();
       }
     } else {
@@ -731,9 +839,6 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
         const int widx = warp - FIRST_RED_WARP;
         const bool active = p.n_items > 0 && (is_gemm ? widx < p.red_warps : true);
         if (active) {
-#ifdef T3_PROFILE
-            long long prof_rwait = 0, prof_rwork = 0, prof_items = 0; const long long prof_start = clock64();
-#endif
 #pragma unroll 1
             while (true) {
                 int t = 0;
@@ -749,10 +854,7 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                 const int ncols_left = min(p.BN, p.N - nt * p.BN) - cc * FRAG_COLS;
                 if (row_base + rib >= p.M || ncols_left <= 0) continue;    // nothing of Y in this item
                 const int region = mt * p.sched.n_nt + nt;
-                PROF_T0(trw);
                 if (!wait_region(p, &p.counters[region], region)) break;
-                PROF_ADD(prof_rwait, trw);
-                PROF_T0(trk);
                 const int slot = p.ring_slots > 0 ? seq % p.ring_slots : region;
                 const size_t chunk_off = static_cast<size_t>(slot) * static_cast<size_t>(p.slot_elems) +
                                          static_cast<size_t>(rb * p.sched.nc + cc) * FRAG_ELEMS;
@@ -760,23 +862,14 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                                         ? static_cast<const void*>(reinterpret_cast<const __nv_bfloat16*>(p.partials) + chunk_off)
                                         : static_cast<const void*>(p.partials + chunk_off);
                 reduce_item(chunk, static_cast<size_t>(p.tile_elems), p.partial_bf16, rib, p.sched.reduce_rows, p.Y, p.M, p.N,
-                            p.R, p.chunk_rows, p.out_f32, row_base, col_base, ncols_left, lane);
+                            p.R, p.chunk_rows, p.out_f32, row_base, col_base, ncols_left, lane, p.epi, p.inplace);
                 if (p.ring_slots > 0) {
                     // every lane's loads of this item have returned (their values were used above)
                     __syncwarp();
                     if (lane == 0) red_release_gpu_add(&p.done[region], 1u);
                 }
-                PROF_ADD(prof_rwork, trk);
-#ifdef T3_PROFILE
-                prof_items++;
-#endif
             }
-#ifdef T3_PROFILE
-            if (lane == 0 && widx == 0) {
-                g_prof[blockIdx.x * 16 + 10] = prof_rwait; g_prof[blockIdx.x * 16 + 11] = prof_rwork;
-                g_prof[blockIdx.x * 16 + 12] = prof_items; g_prof[blockIdx.x * 16 + 13] = clock64() - prof_start;
-            }
-#endif
+            if (lane == 0) atomicMax(&trace_s[2], static_cast<unsigned long long>(globaltimer_ns()));
         }
         __syncwarp();
     }
@@ -795,6 +888,10 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
     }
     // the last CTA to finish re-arms the tracker for the next call
     if (threadIdx.x == 0) {
+        if (p.trace != nullptr) {
+            unsigned long long* t = p.trace + 4ull * blockIdx.x;
+            t[0] = trace_s[0]; t[1] = trace_s[1]; t[2] = trace_s[2]; t[3] = globaltimer_ns();
+        }
         __threadfence();
         const uint32_t done = atomicAdd(&p.ctl[1], 1u);
         if (done == gridDim.x - 1) {
@@ -821,7 +918,7 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
 template <int PARTIAL_BF16>       // compiled once per storage type, so that each keeps two blocks per SM
 __global__ void __launch_bounds__(256, 2) t3_reduce_kernel(const float* __restrict__ partials, void* Y, int M, int N, int R,
                                                            int chunk_rows, int out_f32, int BN, Sched sched,
-                                                           long long slot_elems, int tile_elems) {
+                                                           long long slot_elems, int tile_elems, EpiOps epi, int inplace) {
     constexpr int partial_bf16 = PARTIAL_BF16;
     const int lane = static_cast<int>(threadIdx.x) & 31;
     const long long warps = static_cast<long long>(gridDim.x) * (blockDim.x >> 5);
@@ -841,7 +938,7 @@ __global__ void __launch_bounds__(256, 2) t3_reduce_kernel(const float* __restri
         const void* chunk = partial_bf16 ? static_cast<const void*>(reinterpret_cast<const __nv_bfloat16*>(partials) + chunk_off)
                                          : static_cast<const void*>(partials + chunk_off);
         reduce_item(chunk, static_cast<size_t>(tile_elems), partial_bf16, rib, sched.reduce_rows, Y, M, N, R, chunk_rows,
-                    out_f32, row_base, col_base, ncols_left, lane);
+                    out_f32, row_base, col_base, ncols_left, lane, epi, inplace);
     }
 }
 

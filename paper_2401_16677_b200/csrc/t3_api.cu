@@ -4,9 +4,11 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "../../include/t3.h"
@@ -28,6 +30,16 @@ constexpr bool HAVE_SHARED_FETCH = false;
 int fail(int code) {
     g_last_error = code;
     return code;
+}
+
+// One rank of a multi-process launch (torchrun and the like export WORLD_SIZE / LOCAL_WORLD_SIZE): the
+// kernel variant whose W fetches are multicast TMA loads is for one process on one GPU only.
+bool multi_process_launch() {
+    for (const char* key : {"WORLD_SIZE", "LOCAL_WORLD_SIZE"}) {
+        const char* v = std::getenv(key);
+        if (v && *v && std::atoi(v) != 1) return true;
+    }
+    return false;
 }
 
 struct Geometry {
@@ -76,12 +88,17 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
     t3_chunking_t c;
     std::memset(&c, 0, sizeof c);
     if (in) c = *in;
-    if (c.reserved[0] != 0) return T3_ERR_INVALID_ARG;
+    if (c.reserved[0] != 0 || c.reserved[1] != 0 || c.reserved[2] != 0) return T3_ERR_INVALID_ARG;
+    if (c.reduce != T3_REDUCE_RING && c.reduce != T3_REDUCE_INPLACE) return T3_ERR_INVALID_ARG;
     if (c.order != T3_ORDER_GROUPED && c.order != T3_ORDER_STAGGERED) return T3_ERR_INVALID_ARG;
     if (c.w_layout != T3_W_NK && c.w_layout != T3_W_KN) return T3_ERR_INVALID_ARG;
     if (c.partial_dtype != T3_PARTIAL_F32 && c.partial_dtype != T3_PARTIAL_BF16) return T3_ERR_INVALID_ARG;
     if (c.cluster_ctas != 0 && c.cluster_ctas != 2 && c.cluster_ctas != 4) return T3_ERR_INVALID_ARG;
     if (c.mode < T3_MODE_FUSED || c.mode > T3_MODE_REDUCE_ONLY) return T3_ERR_INVALID_ARG;
+    if (c.split_k == 0) c.split_k = 1;
+    if (c.split_k < 1 || c.split_k > 16) return T3_ERR_INVALID_ARG;
+    if (c.split_k > 1 && c.reduce != T3_REDUCE_INPLACE) return T3_ERR_UNSUPPORTED;
+    if (c.reduce == T3_REDUCE_INPLACE && (c.partial_dtype != T3_PARTIAL_F32 || c.order != T3_ORDER_GROUPED)) return T3_ERR_UNSUPPORTED;
 
     if (c.tile_n == 0) c.tile_n = pick_tile_n(N, c.w_layout == T3_W_KN ? 128 : 32);
     if (c.tile_n < 32 || c.tile_n > 256 || c.tile_n % 32) return T3_ERR_INVALID_ARG;
@@ -90,7 +107,11 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
 
     const int64_t n_mt64 = (M + t3::BMJ - 1) / t3::BMJ;
     const int64_t n_nt64 = (N + c.tile_n - 1) / c.tile_n;
-    if (n_mt64 * n_nt64 * R > (1ll << 30)) return T3_ERR_TOO_LARGE;
+    if (c.split_k > (Kr + t3::BK - 1) / t3::BK) return T3_ERR_INVALID_ARG;     // every producer needs a k-block
+    const int Rv = R * c.split_k;                   // producers per output tile ("virtual slices")
+    const bool inplace = c.reduce == T3_REDUCE_INPLACE;
+    const int copies = inplace ? 1 : R;             // stored tiles per region: one accumulator, or one copy per slice
+    if (n_mt64 * n_nt64 * Rv > (1ll << 30)) return T3_ERR_TOO_LARGE;
     const int n_mt = static_cast<int>(n_mt64), n_nt = static_cast<int>(n_nt64);
 
     if (c.group_tiles < 0) return T3_ERR_INVALID_ARG;
@@ -104,9 +125,9 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
         // two groups, see the ring sizing below) within about half of L2: with many slices a slot is large
         // (R = 16, BN = 256: 4 MB) and a group of 8 would ask for a 100 MB ring (measured: 247 -> 203 us on
         // R = 16, M = 4096, H = 2048 with groups of 4)
-        const int64_t slot_b = static_cast<int64_t>(R) * t3::ROW_BLOCKS * ((c.tile_n + t3::FRAG_COLS - 1) / t3::FRAG_COLS) *
+        const int64_t slot_b = static_cast<int64_t>(copies) * t3::ROW_BLOCKS * ((c.tile_n + t3::FRAG_COLS - 1) / t3::FRAG_COLS) *
                                t3::FRAG_ELEMS * (c.partial_dtype == T3_PARTIAL_BF16 ? 2 : 4);
-        while (c.group_tiles > 1 && ((sm_count + R - 1) / R + 2ll * c.group_tiles) * slot_b > (72ll << 20)) c.group_tiles /= 2;
+        while (c.group_tiles > 1 && ((sm_count + Rv - 1) / Rv + 2ll * c.group_tiles) * slot_b > (72ll << 20)) c.group_tiles /= 2;
     }
     if (c.group_tiles > n_mt) c.group_tiles = n_mt;
 
@@ -114,7 +135,7 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
     {
         // Two pairs per cluster work on jobs j, j + 1 (j even): these must be vertically adjacent tiles of
         // one W tile and one slice, which holds when every schedule group has an even number of row tiles.
-        const bool can4 = HAVE_SHARED_FETCH && c.order == T3_ORDER_GROUPED && n_mt % 2 == 0 && c.group_tiles % 2 == 0 && sm_count >= 4 &&
+        const bool can4 = HAVE_SHARED_FETCH && !multi_process_launch() && c.order == T3_ORDER_GROUPED && n_mt % 2 == 0 && c.group_tiles % 2 == 0 && sm_count >= 4 &&
                           (c.max_ctas == 0 || c.max_ctas >= 4) && c.reducer_ctas % 4 == 0;
         if (c.cluster_ctas == 4 && !can4) return T3_ERR_UNSUPPORTED;
         // Clusters of four fit on fewer SMs (132 of 148 on a B200) but fetch W from L2 once per two pairs;
@@ -153,7 +174,7 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
     g.a_bytes = a_bytes;
     g.b_bytes = b_bytes;
     g.stage_bytes = stage_bytes;
-    g.sched = t3::make_sched(n_mt, n_nt, R, c.group_tiles, c.reduce_rows, c.tile_n);
+    g.sched = t3::make_sched(n_mt, n_nt, Rv, c.group_tiles, c.reduce_rows, c.tile_n);
     if (c.order == T3_ORDER_STAGGERED) {
         // device r's chunk of a step must be whole row tiles
         if ((M / R) % t3::BMJ) return T3_ERR_UNSUPPORTED;
@@ -183,8 +204,9 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
     o.n_jobs = g.sched.n_jobs;
     o.n_regions = g.sched.n_regions;
     // Section 4.2.1: threshold = (tile size) x (updates per element); the unit counted here is one
-    // CTA's 128-row half of the tile, and every one of the R slices updates each element once.
-    o.expected = t3::CTA_PAIR * R + ((c.debug_flags & T3_DEBUG_INFLATE_EXPECTED) ? 1 : 0);
+    // CTA's 128-row half of the tile, and every one of the R slices updates each element once (split_k
+    // times when a slice's product is itself split along k, Section 7.7).
+    o.expected = t3::CTA_PAIR * Rv + ((c.debug_flags & T3_DEBUG_INFLATE_EXPECTED) ? 1 : 0);
     o.group_tiles = c.group_tiles;
     o.grid = grid;
     o.reducer_ctas = c.reducer_ctas;
@@ -199,7 +221,7 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
     o.k_blocks = nkb;
     o.smem_bytes = c.stages * static_cast<int>(stage_bytes) + epi_bytes + red_bytes + 1024;
     g.tile_elems = t3::ROW_BLOCKS * g.sched.nc * t3::FRAG_ELEMS;
-    g.slot_elems = static_cast<int64_t>(R) * g.tile_elems;
+    g.slot_elems = static_cast<int64_t>(copies) * g.tile_elems;
     const int esize = c.partial_dtype == T3_PARTIAL_BF16 ? 2 : 4;
     g.partial_bytes = static_cast<int64_t>(g.sched.n_regions) * g.slot_elems * esize;
     {
@@ -212,7 +234,7 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
         int64_t want = c.ring_slots;
         if (want == 0) {
             want = (64ll << 20) / slot_bytes;      // about half of the 126 MB L2
-            const int64_t in_flight = (2ll * pairs + R - 1) / R + 2ll * c.group_tiles;
+            const int64_t in_flight = (2ll * pairs + Rv - 1) / Rv + 2ll * c.group_tiles;
             if (want < in_flight) want = in_flight;
         }
         if (want < 0) want = 0;                                   // -1: full partial buffers in fused mode too
@@ -227,13 +249,17 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
     o.partial_dtype = c.partial_dtype;
     o.w_layout = c.w_layout;
     o.order = c.order;
+    o.reduce = c.reduce;
+    o.split_k = c.split_k;
     const double sy = dtype == T3_BF16_OUT_F32 ? 4.0 : 2.0;
     const double dM = static_cast<double>(M), dN = static_cast<double>(N), dK = static_cast<double>(K);
     o.workspace_bytes = g.partial_bytes + static_cast<int64_t>(4) * (2 * o.n_regions + 64) +
                         static_cast<int64_t>(g.ring_slots) * g.slot_elems * esize;
     o.flops = 2.0 * dM * dN * dK;
-    o.bytes_gemm = 2.0 * dM * dK + 2.0 * dK * dN + static_cast<double>(esize) * R * dM * dN;
-    o.bytes_reduce = static_cast<double>(esize) * R * dM * dN + sy * dM * dN;
+    // update in place: every producer tile still ships 4 bytes per element (to the L2's reduction units); the
+    // final pass reads the accumulator once, clears it and writes Y
+    o.bytes_gemm = 2.0 * dM * dK + 2.0 * dK * dN + static_cast<double>(esize) * Rv * dM * dN;
+    o.bytes_reduce = inplace ? (8.0 + sy) * dM * dN : static_cast<double>(esize) * R * dM * dN + sy * dM * dN;
     o.bytes_fused = o.bytes_gemm + o.bytes_reduce;
     return T3_OK;
 }
@@ -307,6 +333,13 @@ struct t3_plan_s {
     int32_t* status;
     CUtensorMap tmX, tmW;
     float* ring;          // [ring_slots][R][tile_elems] fp32, fused mode only (NULL: fused mode uses the full buffers)
+    int64_t ring_bytes;   // size of that allocation (the tuner may use fewer slots, never more)
+    unsigned long long* trace;   // [trace_ctas][4] device: per-CTA timestamps of the last fused launch
+    int trace_ctas;
+    int last_fused_grid;  // CTAs of the last fused launch (0: none yet)
+    uint32_t epoch;       // launches made so far
+    t3_chunking_t user_cfg;   // the chunking as the caller gave it (zeros for NULL): the tuner's starting point
+    int smem_optin;
     const void* mapX;
     const void* mapW;
     int ptr_lines_aligned;  // the cached X and W pointers are 128-byte aligned
@@ -384,13 +417,94 @@ int prepare_kernel(int cluster_ctas, int grid, int smem_optin) {
     return max_clusters;
 }
 
-int launch_fused(t3_plan_t pl, void* Y, cudaStream_t st, bool with_reduce) {
-    const Geometry& g = pl->geo;
-    t3::KParams kp;
+// Per-device ordering of t3 kernels.  The fused kernel is persistent and all of its clusters must be
+// resident together, so two of them must never share the GPU: every launch waits (on its stream, not on
+// the host) for an event recorded after the previous launch on that device.
+constexpr int MAX_DEVICES = 64;
+struct DeviceOrder {
+    std::mutex mu;
+    cudaEvent_t ev = nullptr;
+};
+DeviceOrder g_dev_order[MAX_DEVICES];
+
+// RAII: holds the device's mutex; enter() makes `st` wait for the previous t3 launch, leave() records
+// this one.  Inside a stream capture both are skipped (the graph orders its own nodes).
+struct OrderedLaunch {
+    DeviceOrder* d = nullptr;
+    cudaStream_t st;
+    bool capturing = false;
+    OrderedLaunch(int dev, cudaStream_t s) : st(s) {
+        if (dev >= 0 && dev < MAX_DEVICES) d = &g_dev_order[dev];
+        if (d) d->mu.lock();
+    }
+    ~OrderedLaunch() {
+        if (d) d->mu.unlock();
+    }
+    int enter() {
+        if (!d) return T3_OK;
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(st, &cs) != cudaSuccess) {
+            cudaGetLastError();
+            return T3_ERR_CUDA;
+        }
+        capturing = cs != cudaStreamCaptureStatusNone;
+        if (capturing) return T3_OK;
+        if (!d->ev) {
+            if (cudaEventCreateWithFlags(&d->ev, cudaEventDisableTiming) != cudaSuccess) {
+                cudaGetLastError();
+                d->ev = nullptr;
+                return T3_ERR_CUDA;
+            }
+            return T3_OK;                      // first launch on this device: nothing to wait for
+        }
+        if (cudaStreamWaitEvent(st, d->ev, 0) != cudaSuccess) {
+            cudaGetLastError();
+            return T3_ERR_CUDA;
+        }
+        return T3_OK;
+    }
+    int leave() {
+        if (!d || capturing || !d->ev) return T3_OK;
+        if (cudaEventRecord(d->ev, st) != cudaSuccess) {
+            cudaGetLastError();
+            return T3_ERR_CUDA;
+        }
+        return T3_OK;
+    }
+};
+
+t3::EpiOps make_epi(const t3_epilogue_t* e) {
+    t3::EpiOps o;
+    std::memset(&o, 0, sizeof o);
+    if (!e) return o;
+    o.bias = e->bias;
+    o.residual = e->residual;
+    o.keep = static_cast<const uint8_t*>(e->keep);
+    o.keep_scale = e->keep_scale;
+    o.bias_f32 = e->bias_dtype == T3_EPI_F32;
+    o.residual_f32 = e->residual_dtype == T3_EPI_F32;
+    o.any = (o.bias || o.residual || o.keep) ? 1 : 0;
+    return o;
+}
+
+int check_epi(const t3_epilogue_t* e, const void* Y) {
+    if (!e) return T3_OK;
+    if (e->reserved != 0) return T3_ERR_INVALID_ARG;
+    if ((e->bias_dtype != T3_EPI_BF16 && e->bias_dtype != T3_EPI_F32) ||
+        (e->residual_dtype != T3_EPI_BF16 && e->residual_dtype != T3_EPI_F32))
+        return T3_ERR_INVALID_ARG;
+    if ((reinterpret_cast<uintptr_t>(e->bias) | reinterpret_cast<uintptr_t>(e->residual) | reinterpret_cast<uintptr_t>(e->keep)) & 15u)
+        return T3_ERR_INVALID_ARG;
+    if (e->residual && e->residual == Y) return T3_ERR_INVALID_ARG;
+    return T3_OK;
+}
+
+// Kernel parameters of geometry `g` over the plan's buffers.
+void fill_params(t3_plan_t pl, const Geometry& g, void* Y, bool with_reduce, const t3::EpiOps& epi, t3::KParams& kp) {
     std::memset(&kp, 0, sizeof kp);
     kp.tmX = pl->tmX;
     kp.tmW = pl->tmW;
-    const bool use_ring = with_reduce && pl->ring != nullptr;
+    const bool use_ring = with_reduce && pl->ring != nullptr && g.ring_slots > 0;
     kp.ring_slots = use_ring ? g.ring_slots : 0;
     kp.slot_elems = g.slot_elems;
     kp.tile_elems = g.tile_elems;
@@ -422,24 +536,73 @@ int launch_fused(t3_plan_t pl, void* Y, cudaStream_t st, bool with_reduce) {
     kp.out_f32 = g.info.dtype == T3_BF16_OUT_F32;
     kp.expected = static_cast<uint32_t>(g.info.expected);
     kp.timeout_ns = static_cast<unsigned long long>(g.cfg.timeout_ms) * 1000000ull;
+    kp.inplace = g.cfg.reduce == T3_REDUCE_INPLACE;
+    kp.split_k = g.info.split_k;
+    kp.epi = epi;
+    kp.trace = (with_reduce && g.info.grid <= pl->trace_ctas) ? pl->trace : nullptr;
+}
+
+int launch_fused(t3_plan_t pl, const Geometry& g, void* Y, cudaStream_t st, bool with_reduce, const t3::EpiOps& epi) {
+    t3::KParams kp;
+    fill_params(pl, g, Y, with_reduce, epi, kp);
+    kp.epoch = ++pl->epoch;
+    if (kp.epoch == 0) kp.epoch = ++pl->epoch;        // 0 is "nobody is aborting"
+    if (kp.trace) pl->last_fused_grid = g.info.grid;
     return launch_kernel(kp, g.info.cluster_ctas, g.info.grid, g.info.smem_bytes, st);
 }
 
-int launch_reduce(t3_plan_t pl, void* Y, cudaStream_t st) {
-    const Geometry& g = pl->geo;
+int launch_reduce(t3_plan_t pl, const Geometry& g, void* Y, cudaStream_t st, const t3::EpiOps& epi) {
     const t3_info_t& o = g.info;
     long long blocks = (static_cast<long long>(o.n_reduce_items) + 7) / 8;      // 8 warps per block, one item each
     const long long cap = static_cast<long long>(pl->sm_count) * 8;
     if (blocks > cap) blocks = cap;
+    const int inplace = g.cfg.reduce == T3_REDUCE_INPLACE;
     if (g.cfg.partial_dtype == T3_PARTIAL_BF16)
         t3::t3_reduce_kernel<1><<<static_cast<unsigned>(blocks), 256, 0, st>>>(
             pl->partials, Y, static_cast<int>(o.M), static_cast<int>(o.N), o.R, o.chunk_rows,
-            o.dtype == T3_BF16_OUT_F32, o.tile_n, g.sched, g.slot_elems, g.tile_elems);
+            o.dtype == T3_BF16_OUT_F32, o.tile_n, g.sched, g.slot_elems, g.tile_elems, epi, inplace);
     else
         t3::t3_reduce_kernel<0><<<static_cast<unsigned>(blocks), 256, 0, st>>>(
             pl->partials, Y, static_cast<int>(o.M), static_cast<int>(o.N), o.R, o.chunk_rows,
-            o.dtype == T3_BF16_OUT_F32, o.tile_n, g.sched, g.slot_elems, g.tile_elems);
+            o.dtype == T3_BF16_OUT_F32, o.tile_n, g.sched, g.slot_elems, g.tile_elems, epi, inplace);
     return cudaGetLastError() == cudaSuccess ? T3_OK : T3_ERR_CUDA;
+}
+
+// Every cluster must be resident at once (reducers wait on tiles that other pairs produce): sets the
+// kernel's shared-memory attribute and shrinks the grid to what the device can hold.
+int fit_to_device(Geometry& g, int smem_optin) {
+    t3_info_t& oi = g.info;
+    if (oi.smem_bytes + SMEM_STATIC_SLACK > smem_optin) return T3_ERR_CUDA;
+    const int cl = oi.cluster_ctas;
+    const int max_clusters = prepare_kernel(cl, oi.grid, smem_optin);
+    if (max_clusters < 1) return T3_ERR_CUDA;
+    if (oi.grid > cl * max_clusters) {
+        const int new_grid = cl * max_clusters;
+        if (oi.reducer_ctas >= new_grid) return T3_ERR_UNSUPPORTED;
+        oi.gemm_ctas = new_grid - oi.reducer_ctas;
+        if (oi.gemm_ctas > t3::CTA_PAIR * oi.n_jobs) oi.gemm_ctas = t3::CTA_PAIR * oi.n_jobs;
+        oi.grid = oi.gemm_ctas + oi.reducer_ctas;
+    }
+    return T3_OK;
+}
+
+// One call in `mode` with geometry `g`, ordered after the device's previous t3 launch.
+int run_mode(t3_plan_t pl, const Geometry& g, int mode, void* Y, cudaStream_t st, const t3::EpiOps& epi) {
+    OrderedLaunch ord(pl->device, st);
+    int rc = ord.enter();
+    if (rc != T3_OK) return rc;
+    switch (mode) {
+        case T3_MODE_FUSED: rc = launch_fused(pl, g, Y, st, true, epi); break;
+        case T3_MODE_GEMM_ONLY: rc = launch_fused(pl, g, Y, st, false, epi); break;
+        case T3_MODE_SEQUENTIAL:
+            rc = launch_fused(pl, g, Y, st, false, epi);
+            if (rc == T3_OK) rc = launch_reduce(pl, g, Y, st, epi);
+            break;
+        case T3_MODE_REDUCE_ONLY: rc = launch_reduce(pl, g, Y, st, epi); break;
+        default: rc = T3_ERR_INVALID_ARG;
+    }
+    const int rc2 = ord.leave();
+    return rc != T3_OK ? rc : rc2;
 }
 
 }  // namespace
@@ -550,32 +713,15 @@ t3_plan_t t3_plan(int64_t M, int64_t N, int64_t K, int32_t R, t3_dtype_t dtype, 
     }
     pl->device = dev;
     pl->sm_count = prop.multiProcessorCount;
+    pl->smem_optin = static_cast<int>(prop.sharedMemPerBlockOptin);
+    if (chunking) pl->user_cfg = *chunking;
     const t3_info_t& o = pl->geo.info;
-    if (o.smem_bytes + SMEM_STATIC_SLACK > static_cast<int>(prop.sharedMemPerBlockOptin)) {
-        delete pl;
-        fail(T3_ERR_CUDA);
-        return nullptr;
-    }
     {
-        // every cluster must be resident at once: reducers wait on tiles that other pairs produce
-        const int cl = o.cluster_ctas;
-        const int max_clusters = prepare_kernel(cl, o.grid, static_cast<int>(prop.sharedMemPerBlockOptin));
-        if (max_clusters < 1) {
+        const int rc2 = fit_to_device(pl->geo, static_cast<int>(prop.sharedMemPerBlockOptin));
+        if (rc2 != T3_OK) {
             delete pl;
-            fail(T3_ERR_CUDA);
+            fail(rc2);
             return nullptr;
-        }
-        t3_info_t& oi = pl->geo.info;
-        if (oi.grid > cl * max_clusters) {
-            const int new_grid = cl * max_clusters;
-            if (oi.reducer_ctas >= new_grid) {
-                delete pl;
-                fail(T3_ERR_UNSUPPORTED);
-                return nullptr;
-            }
-            oi.gemm_ctas = new_grid - oi.reducer_ctas;
-            if (oi.gemm_ctas > t3::CTA_PAIR * oi.n_jobs) oi.gemm_ctas = t3::CTA_PAIR * oi.n_jobs;
-            oi.grid = oi.gemm_ctas + oi.reducer_ctas;
         }
     }
     const size_t pbytes = static_cast<size_t>(pl->geo.partial_bytes);
@@ -605,6 +751,22 @@ t3_plan_t t3_plan(int64_t M, int64_t N, int64_t K, int32_t R, t3_dtype_t dtype, 
             fail(T3_ERR_ALLOC);
             return nullptr;
         }
+        pl->ring_bytes = static_cast<int64_t>(rbytes);
+    }
+    if (pl->geo.cfg.reduce == T3_REDUCE_INPLACE) {
+        // accumulator tiles start at zero; every call's final pass leaves them at zero again
+        cudaMemset(pl->partials, 0, pbytes);
+        if (pl->ring) cudaMemset(pl->ring, 0, static_cast<size_t>(pl->ring_bytes));
+    }
+    pl->trace_ctas = pl->sm_count;
+    if (cudaMalloc(&pl->trace, static_cast<size_t>(pl->trace_ctas) * 4 * sizeof(unsigned long long)) != cudaSuccess) {
+        cudaGetLastError();
+        cudaFree(pl->partials);
+        cudaFree(pl->counters);
+        cudaFree(pl->ring);
+        delete pl;
+        fail(T3_ERR_ALLOC);
+        return nullptr;
     }
     pl->done = pl->counters + o.n_regions;
     pl->ctl = pl->counters + 2 * o.n_regions;
@@ -613,7 +775,12 @@ t3_plan_t t3_plan(int64_t M, int64_t N, int64_t K, int32_t R, t3_dtype_t dtype, 
     return pl;
 }
 
-int t3_gemm_rs_mode(t3_plan_t pl, int32_t mode, const void* X, const void* W, void* Y, void* stream) {
+}  // extern "C"
+
+namespace {
+
+// Validation, tensor maps and the launch shared by t3_gemm_rs, t3_gemm_rs_mode and t3_gemm_rs_ex.
+int gemm_rs_common(t3_plan_t pl, int32_t mode, const void* X, const void* W, void* Y, const t3_epilogue_t* epi, void* stream) {
     if (!valid(pl)) return fail(T3_ERR_INVALID_ARG);
     if (mode < T3_MODE_FUSED || mode > T3_MODE_REDUCE_ONLY) return fail(T3_ERR_INVALID_ARG);
     const bool need_in = mode != T3_MODE_REDUCE_ONLY;
@@ -621,11 +788,18 @@ int t3_gemm_rs_mode(t3_plan_t pl, int32_t mode, const void* X, const void* W, vo
     if ((need_in && (!X || !W)) || (need_out && !Y)) return fail(T3_ERR_INVALID_ARG);
     if ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W) | reinterpret_cast<uintptr_t>(Y)) & 15u)
         return fail(T3_ERR_INVALID_ARG);
+    int rc = check_epi(epi, Y);
+    if (rc != T3_OK) return fail(rc);
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev != pl->device) {
+        cudaGetLastError();
+        return fail(T3_ERR_DEVICE);
+    }
     const t3_info_t& o = pl->geo.info;
     if (mode == T3_MODE_FUSED && o.reducer_warps == 0 && o.reducer_ctas == 0) return fail(T3_ERR_UNSUPPORTED);
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (need_in && (X != pl->mapX || W != pl->mapW)) {
-        int rc = encode_sliced_map(&pl->tmX, X, o.M, o.K, o.R, t3::BM);
+        rc = encode_sliced_map(&pl->tmX, X, o.M, o.K, o.R, t3::BM);
         if (rc == T3_OK) rc = encode_w_map(&pl->tmW, W, o);
         if (rc != T3_OK) {
             pl->mapX = pl->mapW = nullptr;
@@ -636,22 +810,26 @@ int t3_gemm_rs_mode(t3_plan_t pl, int32_t mode, const void* X, const void* W, vo
         pl->ptr_lines_aligned = ((reinterpret_cast<uintptr_t>(X) | reinterpret_cast<uintptr_t>(W)) & 127u) == 0;
     }
     pl->last_stream = st;
-    int rc = T3_OK;
-    switch (mode) {
-        case T3_MODE_FUSED: rc = launch_fused(pl, Y, st, true); break;
-        case T3_MODE_GEMM_ONLY: rc = launch_fused(pl, Y, st, false); break;
-        case T3_MODE_SEQUENTIAL:
-            rc = launch_fused(pl, Y, st, false);
-            if (rc == T3_OK) rc = launch_reduce(pl, Y, st);
-            break;
-        case T3_MODE_REDUCE_ONLY: rc = launch_reduce(pl, Y, st); break;
-    }
+    rc = run_mode(pl, pl->geo, mode, Y, st, make_epi(epi));
     return rc == T3_OK ? T3_OK : fail(rc);
+}
+
+}  // namespace
+
+extern "C" {
+
+int t3_gemm_rs_mode(t3_plan_t pl, int32_t mode, const void* X, const void* W, void* Y, void* stream) {
+    return gemm_rs_common(pl, mode, X, W, Y, nullptr, stream);
 }
 
 int t3_gemm_rs(t3_plan_t pl, const void* X, const void* W, void* Y, void* stream) {
     if (!valid(pl)) return fail(T3_ERR_INVALID_ARG);
-    return t3_gemm_rs_mode(pl, pl->geo.cfg.mode, X, W, Y, stream);
+    return gemm_rs_common(pl, pl->geo.cfg.mode, X, W, Y, nullptr, stream);
+}
+
+int t3_gemm_rs_ex(t3_plan_t pl, const void* X, const void* W, void* Y, const t3_epilogue_t* epi, void* stream) {
+    if (!valid(pl)) return fail(T3_ERR_INVALID_ARG);
+    return gemm_rs_common(pl, pl->geo.cfg.mode, X, W, Y, epi, stream);
 }
 
 int t3_gemm_rs_host(t3_plan_t pl, const void* Xh, const void* Wh, void* Yh, void* stream) {
@@ -719,8 +897,48 @@ int t3_plan_partials(t3_plan_t pl, void** partials, int64_t* bytes) {
     return T3_OK;
 }
 
+int t3_plan_ring(t3_plan_t pl, void** ring, int64_t* bytes) {
+    if (!valid(pl) || !ring) return fail(T3_ERR_INVALID_ARG);
+    *ring = pl->ring;
+    if (bytes) *bytes = pl->ring ? pl->ring_bytes : 0;
+    return T3_OK;
+}
+
+int t3_plan_timeline(t3_plan_t pl, t3_timeline_t* out) {
+    if (!valid(pl) || !out) return fail(T3_ERR_INVALID_ARG);
+    std::memset(out, 0, sizeof *out);
+    if (pl->last_fused_grid <= 0) return fail(T3_ERR_UNSUPPORTED);       // no fused call yet
+    if (cudaStreamSynchronize(pl->last_stream) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(T3_ERR_CUDA);
+    }
+    const int n = pl->last_fused_grid;
+    unsigned long long h[4 * 160];
+    if (n > 160 || cudaMemcpy(h, pl->trace, static_cast<size_t>(n) * 4 * sizeof(unsigned long long), cudaMemcpyDeviceToHost) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(T3_ERR_CUDA);
+    }
+    unsigned long long t0 = ~0ull, t_pub = 0, t_red = 0, t_end = 0;
+    for (int i = 0; i < n; ++i) {
+        t0 = std::min(t0, h[4 * i]);
+        t_pub = std::max(t_pub, h[4 * i + 1]);
+        t_red = std::max(t_red, h[4 * i + 2]);
+        t_end = std::max(t_end, h[4 * i + 3]);
+    }
+    if (t_pub < t0) t_pub = t0;
+    if (t_red < t_pub) t_red = t_pub;
+    if (t_end < t_red) t_end = t_red;
+    out->total_us = 1e-3 * static_cast<double>(t_end - t0);
+    out->produce_us = 1e-3 * static_cast<double>(t_pub - t0);
+    out->tail_us = 1e-3 * static_cast<double>(t_red - t_pub);
+    out->drain_us = 1e-3 * static_cast<double>(t_end - t_red);
+    out->ctas = n;
+    return T3_OK;
+}
+
 int t3_plan_export_partials(t3_plan_t pl, void* dst, void* stream) {
     if (!valid(pl) || !dst || (reinterpret_cast<uintptr_t>(dst) & 3u)) return fail(T3_ERR_INVALID_ARG);
+    if (pl->geo.cfg.reduce == T3_REDUCE_INPLACE) return fail(T3_ERR_UNSUPPORTED);
     const Geometry& g = pl->geo;
     const t3_info_t& o = g.info;
     const long long total = static_cast<long long>(o.R) * o.M * o.N;
@@ -754,6 +972,11 @@ int t3_plan_status(t3_plan_t pl, t3_status_t* out) {
         // has already re-armed the tracker counters)
         cudaMemset(pl->status, 0, sizeof h);
         cudaMemset(pl->counters, 0, static_cast<size_t>(4) * (2 * pl->geo.info.n_regions + 8));
+        if (pl->geo.cfg.reduce == T3_REDUCE_INPLACE) {
+            // half-accumulated tiles of the aborted call
+            cudaMemset(pl->partials, 0, static_cast<size_t>(pl->geo.partial_bytes));
+            if (pl->ring) cudaMemset(pl->ring, 0, static_cast<size_t>(pl->ring_bytes));
+        }
         return fail(h[0]);
     }
     return T3_OK;
@@ -776,14 +999,17 @@ struct StaticDeviceState {
     int sm_count;
     int cc_major;
     int max_clusters;     // resident CTA pairs of the fused kernel at its largest shared-memory size
+    int smem_optin;       // opt-in shared memory per block
 };
 StaticDeviceState g_static_dev[MAX_STATIC_DEVICES];   // zero-initialised; written once per device
+std::once_flag g_static_once[MAX_STATIC_DEVICES];
 
-// Once per device, with that device current.
+// Once per device, with that device current; host threads making their first calls together meet in
+// std::call_once, so each sees the fields complete.
 int static_device_setup(int dev, StaticDeviceState** out) {
     if (dev < 0 || dev >= MAX_STATIC_DEVICES) return T3_ERR_DEVICE;
     StaticDeviceState& st = g_static_dev[dev];
-    if (st.ready == 0) {
+    std::call_once(g_static_once[dev], [&st, dev]() {
         int rc = 1;
         void* ptr = nullptr;
         int sms = 0, major = 0, smem_optin = 0;
@@ -806,10 +1032,11 @@ int static_device_setup(int dev, StaticDeviceState** out) {
                 st.sm_count = sms;
                 st.cc_major = major;
                 st.max_clusters = mc;
+                st.smem_optin = smem_optin;
             }
         }
         st.ready = rc;
-    }
+    });
     if (st.ready != 1) return st.ready;
     *out = &st;
     return T3_OK;
@@ -842,6 +1069,7 @@ int t3_gemm_rs_static(int64_t M, int64_t N, int64_t K, int32_t R, t3_dtype_t dty
     rc = resolve_geometry(M, N, K, R, static_cast<int>(dtype), &ch, st->sm_count, g);
     if (rc != T3_OK) return fail(rc);
     t3_info_t& o = g.info;
+    if (o.smem_bytes + SMEM_STATIC_SLACK > st->smem_optin) return fail(T3_ERR_CUDA);
     if (o.grid > t3::CTA_PAIR * st->max_clusters) {          // every pair must be resident at once
         o.gemm_ctas = t3::CTA_PAIR * st->max_clusters;
         if (o.gemm_ctas > t3::CTA_PAIR * o.n_jobs) o.gemm_ctas = t3::CTA_PAIR * o.n_jobs;
@@ -888,6 +1116,8 @@ int t3_gemm_rs_static(int64_t M, int64_t N, int64_t K, int32_t R, t3_dtype_t dty
     kp.out_f32 = dtype == T3_BF16_OUT_F32;
     kp.expected = static_cast<uint32_t>(o.expected);
     kp.timeout_ns = static_cast<unsigned long long>(g.cfg.timeout_ms) * 1000000ull;
+    kp.split_k = 1;
+    kp.epoch = 1;             // the tracker words, ctl[2] among them, are cleared before every launch
 
     cudaStream_t cs = static_cast<cudaStream_t>(stream);
     // the array keeps whatever the previous call left: the tracker must start at zero
@@ -899,11 +1129,122 @@ int t3_gemm_rs_static(int64_t M, int64_t N, int64_t K, int32_t R, t3_dtype_t dty
     return T3_OK;
 }
 
-#ifdef T3_PROFILE
-int t3_debug_read_profile(long long* out, int n) {
-    return cudaMemcpyFromSymbol(out, t3::g_prof, sizeof(long long) * n) == cudaSuccess ? 0 : -1;
+int t3_plan_tune(t3_plan_t pl, const void* X, const void* W, void* Y, void* stream, t3_tune_t* out) {
+    if (!valid(pl) || !X || !W || !Y) return fail(T3_ERR_INVALID_ARG);
+    if (out) std::memset(out, 0, sizeof *out);
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    {
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (cudaStreamIsCapturing(st, &cs) != cudaSuccess || cs != cudaStreamCaptureStatusNone) {
+            cudaGetLastError();
+            return fail(T3_ERR_UNSUPPORTED);
+        }
+    }
+    if (pl->geo.cfg.mode != T3_MODE_FUSED) return T3_OK;        // the caller fixed the mode: nothing to choose
+    // a first ordinary call: validates the pointers and the device, encodes the tensor maps
+    int rc = gemm_rs_common(pl, T3_MODE_FUSED, X, W, Y, nullptr, stream);
+    if (rc != T3_OK) return rc;
+    t3_status_t stt;
+    rc = t3_plan_status(pl, &stt);
+    if (rc != T3_OK) return rc;
+
+    const Geometry cur = pl->geo;
+    const t3_info_t& o = cur.info;
+    const int esize = cur.cfg.partial_dtype == T3_PARTIAL_BF16 ? 2 : 4;
+    const int64_t slot_bytes = cur.slot_elems * esize;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) {
+        cudaGetLastError();
+        if (e0) cudaEventDestroy(e0);
+        return fail(T3_ERR_CUDA);
+    }
+    constexpr int MAX_CAND = 48, TIMED = 5;
+    Geometry best = cur;
+    float best_us = 0.f, cur_us = 0.f;
+    int n = 0, chosen = 0;
+    const int kinds[3] = {0, 1, 2};                 // fused + ring, fused + full buffers, sequential
+    const int rrs[2] = {cur.cfg.reduce_rows, cur.cfg.reduce_rows == 32 ? 16 : 32};
+    const int cls[2] = {o.cluster_ctas, o.cluster_ctas == 2 ? 4 : 2};
+    const int gts[2] = {o.group_tiles, o.group_tiles / 2};
+    const t3::EpiOps no_epi = make_epi(nullptr);
+    for (int ki = 0; ki < 3; ++ki)
+        for (int ri = 0; ri < 2; ++ri)
+            for (int ci = 0; ci < 2; ++ci)
+                for (int gi = 0; gi < 2; ++gi) {
+                    if (n >= MAX_CAND) break;
+                    if (gts[gi] < 1 || (gi == 1 && gts[1] == gts[0])) continue;
+                    t3_chunking_t c = pl->user_cfg;
+                    c.tile_n = o.tile_n;                      // the workspace is laid out for this tile width
+                    c.mode = kinds[ki] == 2 ? T3_MODE_SEQUENTIAL : T3_MODE_FUSED;
+                    c.reduce_rows = rrs[ri];
+                    c.cluster_ctas = cls[ci];
+                    c.group_tiles = gts[gi];
+                    if (kinds[ki] == 0) {
+                        if (!pl->ring) continue;
+                        c.ring_slots = pl->user_cfg.ring_slots > 0 ? pl->user_cfg.ring_slots : 0;
+                    } else {
+                        c.ring_slots = -1;
+                    }
+                    Geometry g;
+                    if (resolve_geometry(o.M, o.N, o.K, o.R, o.dtype, &c, pl->sm_count, g) != T3_OK) continue;
+                    if (kinds[ki] == 0) {
+                        if (g.ring_slots == 0) continue;      // resolves to full buffers: same as kind 1
+                        if (g.ring_slots * slot_bytes > pl->ring_bytes) {
+                            c.ring_slots = static_cast<int32_t>(pl->ring_bytes / slot_bytes);   // what is allocated
+                            if (c.ring_slots < c.group_tiles ||
+                                resolve_geometry(o.M, o.N, o.K, o.R, o.dtype, &c, pl->sm_count, g) != T3_OK || g.ring_slots == 0)
+                                continue;
+                        }
+                    }
+                    if (g.info.tile_n != o.tile_n || g.partial_bytes != cur.partial_bytes) continue;
+                    if (fit_to_device(g, pl->smem_optin) != T3_OK) continue;
+                    // one untimed call, then TIMED timed ones
+                    float us[TIMED];
+                    bool ok = run_mode(pl, g, c.mode, Y, st, no_epi) == T3_OK;
+                    for (int t = 0; ok && t < TIMED; ++t) {
+                        ok = cudaEventRecord(e0, st) == cudaSuccess && run_mode(pl, g, c.mode, Y, st, no_epi) == T3_OK &&
+                             cudaEventRecord(e1, st) == cudaSuccess && cudaEventSynchronize(e1) == cudaSuccess;
+                        float ms = 0.f;
+                        ok = ok && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess;
+                        us[t] = 1e3f * ms;
+                    }
+                    pl->last_stream = st;
+                    if (!ok || t3_plan_status(pl, &stt) != T3_OK) {
+                        cudaGetLastError();
+                        continue;
+                    }
+                    std::sort(us, us + TIMED);
+                    const float med = us[TIMED / 2];
+                    if (out) {
+                        out->mode[n] = c.mode; out->ring_slots[n] = g.ring_slots; out->reduce_rows[n] = g.info.reduce_rows;
+                        out->cluster_ctas[n] = g.info.cluster_ctas; out->group_tiles[n] = g.info.group_tiles; out->us[n] = med;
+                    }
+                    if (n == 0) cur_us = med;                 // the first candidate is the current configuration
+                    if (n == 0 || med < best_us) {
+                        best_us = med;
+                        best = g;
+                        chosen = n;
+                    }
+                    ++n;
+                }
+    cudaEventDestroy(e0);
+    cudaEventDestroy(e1);
+    if (n == 0) return fail(T3_ERR_CUDA);
+    // keep the current configuration unless the best candidate is at least 2 % faster
+    if (chosen != 0 && best_us > 0.98f * cur_us) {
+        best = cur;
+        chosen = 0;
+    }
+    pl->geo = best;
+    pl->geo.info.tuned = 1;
+    pl->geo.info.mode = pl->geo.cfg.mode;
+    if (out) {
+        out->n_tried = n;
+        out->chosen = chosen;
+    }
+    // leave Y written by the chosen configuration
+    return gemm_rs_common(pl, pl->geo.cfg.mode, X, W, Y, nullptr, stream);
 }
-#endif
 
 int t3_destroy(t3_plan_t pl) {
     if (!pl) return T3_OK;
@@ -913,6 +1254,7 @@ int t3_destroy(t3_plan_t pl) {
     cudaFree(pl->partials);
     cudaFree(pl->ring);
     cudaFree(pl->counters);
+    cudaFree(pl->trace);
     release_host_path(pl);
     pl->magic = 0;
     delete pl;

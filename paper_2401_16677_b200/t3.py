@@ -57,11 +57,14 @@ MODE_FUSED, MODE_SEQUENTIAL, MODE_GEMM_ONLY, MODE_REDUCE_ONLY = 0, 1, 2, 3
 PARTIAL_F32, PARTIAL_BF16 = 0, 1
 W_NK, W_KN = 0, 1
 ORDER_GROUPED, ORDER_STAGGERED = 0, 1
+REDUCE_RING, REDUCE_INPLACE = 0, 1
+EPI_BF16, EPI_F32 = 0, 1
 DEBUG_INFLATE_EXPECTED = 1
 
 EXPORTS = [
-    "t3_plan", "t3_gemm_rs", "t3_gemm_rs_mode", "t3_gemm_rs_host", "t3_gemm_rs_static", "t3_destroy", "t3_plan_info", "t3_plan_status",
-    "t3_plan_partials", "t3_plan_export_partials", "t3_geometry", "t3_schedule", "t3_reduce_schedule", "t3_ring_order",
+    "t3_plan", "t3_gemm_rs", "t3_gemm_rs_mode", "t3_gemm_rs_ex", "t3_gemm_rs_host", "t3_gemm_rs_static", "t3_destroy",
+    "t3_plan_info", "t3_plan_status", "t3_plan_tune", "t3_plan_timeline",
+    "t3_plan_partials", "t3_plan_ring", "t3_plan_export_partials", "t3_geometry", "t3_schedule", "t3_reduce_schedule", "t3_ring_order",
     "t3_last_error", "t3_strerror", "t3_version", "t3_shared_fetch_available",
 ]
 
@@ -72,8 +75,37 @@ class Chunking(ctypes.Structure):
         ("reducer_ctas", ctypes.c_int32), ("reducer_warps", ctypes.c_int32), ("reduce_rows", ctypes.c_int32),
         ("stages", ctypes.c_int32), ("timeout_ms", ctypes.c_int32), ("debug_flags", ctypes.c_int32),
         ("max_ctas", ctypes.c_int32), ("ring_slots", ctypes.c_int32), ("cluster_ctas", ctypes.c_int32),
-        ("partial_dtype", ctypes.c_int32), ("w_layout", ctypes.c_int32), ("order", ctypes.c_int32), ("reserved", ctypes.c_int32 * 1),
+        ("partial_dtype", ctypes.c_int32), ("w_layout", ctypes.c_int32), ("order", ctypes.c_int32),
+        ("reduce", ctypes.c_int32), ("split_k", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3),
     ]
+
+
+class Epilogue(ctypes.Structure):
+    """t3_epilogue_t: element-wise work fused on the reduced chunk (device pointers; 0 = skip)."""
+    _fields_ = [
+        ("bias", ctypes.c_void_p), ("residual", ctypes.c_void_p), ("keep", ctypes.c_void_p),
+        ("keep_scale", ctypes.c_float), ("bias_dtype", ctypes.c_int32), ("residual_dtype", ctypes.c_int32),
+        ("reserved", ctypes.c_int32),
+    ]
+
+
+class Timeline(ctypes.Structure):
+    _fields_ = [("total_us", ctypes.c_double), ("produce_us", ctypes.c_double), ("tail_us", ctypes.c_double),
+                ("drain_us", ctypes.c_double), ("ctas", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+    def as_dict(self) -> dict:
+        return {n: getattr(self, n) for n, _ in self._fields_ if n != "reserved"}
+
+
+class Tune(ctypes.Structure):
+    _fields_ = [("n_tried", ctypes.c_int32), ("chosen", ctypes.c_int32),
+                ("mode", ctypes.c_int32 * 48), ("ring_slots", ctypes.c_int32 * 48), ("reduce_rows", ctypes.c_int32 * 48),
+                ("cluster_ctas", ctypes.c_int32 * 48), ("group_tiles", ctypes.c_int32 * 48), ("us", ctypes.c_float * 48)]
+
+    def candidates(self) -> list:
+        return [dict(mode=self.mode[i], ring_slots=self.ring_slots[i], reduce_rows=self.reduce_rows[i],
+                     cluster_ctas=self.cluster_ctas[i], group_tiles=self.group_tiles[i], us=float(self.us[i]))
+                for i in range(self.n_tried)]
 
 
 class Info(ctypes.Structure):
@@ -90,6 +122,7 @@ class Info(ctypes.Structure):
         ("stages", ctypes.c_int32), ("k_blocks", ctypes.c_int32), ("smem_bytes", ctypes.c_int32),
         ("mode", ctypes.c_int32), ("dtype", ctypes.c_int32), ("cluster_ctas", ctypes.c_int32),
         ("partial_dtype", ctypes.c_int32), ("w_layout", ctypes.c_int32), ("order", ctypes.c_int32),
+        ("reduce", ctypes.c_int32), ("split_k", ctypes.c_int32), ("tuned", ctypes.c_int32), ("reserved0", ctypes.c_int32),
         ("workspace_bytes", ctypes.c_int64),
         ("flops", ctypes.c_double), ("bytes_gemm", ctypes.c_double), ("bytes_reduce", ctypes.c_double),
         ("bytes_fused", ctypes.c_double),
@@ -129,6 +162,14 @@ def lib() -> ctypes.CDLL:
         L.t3_gemm_rs.restype = ctypes.c_int
         L.t3_gemm_rs_mode.argtypes = [p, i32, p, p, p, p]
         L.t3_gemm_rs_mode.restype = ctypes.c_int
+        L.t3_gemm_rs_ex.argtypes = [p, p, p, p, ctypes.POINTER(Epilogue), p]
+        L.t3_gemm_rs_ex.restype = ctypes.c_int
+        L.t3_plan_tune.argtypes = [p, p, p, p, p, ctypes.POINTER(Tune)]
+        L.t3_plan_tune.restype = ctypes.c_int
+        L.t3_plan_timeline.argtypes = [p, ctypes.POINTER(Timeline)]
+        L.t3_plan_timeline.restype = ctypes.c_int
+        L.t3_plan_ring.argtypes = [p, ctypes.POINTER(ctypes.c_void_p), ctypes.POINTER(ctypes.c_int64)]
+        L.t3_plan_ring.restype = ctypes.c_int
         L.t3_gemm_rs_host.argtypes = [p, p, p, p, p]
         L.t3_gemm_rs_host.restype = ctypes.c_int
         L.t3_gemm_rs_static.argtypes = [i64, i64, i64, i32, i32, p, p, p, p]
@@ -185,6 +226,14 @@ def gemm_rs_static(M: int, N: int, K: int, R: int, dtype: int, X: int, W: int, Y
     rc = lib().t3_gemm_rs_static(M, N, K, R, dtype, X, W, Y, stream)
     if rc != OK:
         raise T3Error(rc, "t3_gemm_rs_static")
+
+
+def epilogue(bias: int = 0, residual: int = 0, keep: int = 0, keep_scale: float = 1.0,
+             bias_dtype: int = EPI_BF16, residual_dtype: int = EPI_BF16) -> Epilogue:
+    e = Epilogue()
+    e.bias, e.residual, e.keep = bias or None, residual or None, keep or None
+    e.keep_scale, e.bias_dtype, e.residual_dtype = float(keep_scale), int(bias_dtype), int(residual_dtype)
+    return e
 
 
 def chunking(**kw) -> Chunking:
@@ -267,6 +316,37 @@ class Plan:
         rc = lib().t3_gemm_rs_mode(self._h, mode, X, W, Y, stream)
         if rc != OK:
             raise T3Error(rc, "t3_gemm_rs_mode")
+
+    def gemm_rs_ex(self, X: int, W: int, Y: int, epi: Optional[Epilogue], stream: int = 0) -> None:
+        """t3_gemm_rs with bias / dropout mask / residual fused on the reduced chunk."""
+        rc = lib().t3_gemm_rs_ex(self._h, X, W, Y, ctypes.byref(epi) if epi is not None else None, stream)
+        if rc != OK:
+            raise T3Error(rc, "t3_gemm_rs_ex")
+
+    def tune(self, X: int, W: int, Y: int, stream: int = 0) -> Tune:
+        """t3_plan_tune: short trial on the real operands; keeps the fastest configuration."""
+        out = Tune()
+        rc = lib().t3_plan_tune(self._h, X, W, Y, stream, ctypes.byref(out))
+        if rc != OK:
+            raise T3Error(rc, "t3_plan_tune")
+        return out
+
+    def timeline(self) -> Timeline:
+        """t3_plan_timeline of the last fused call (synchronises)."""
+        out = Timeline()
+        rc = lib().t3_plan_timeline(self._h, ctypes.byref(out))
+        if rc != OK:
+            raise T3Error(rc, "t3_plan_timeline")
+        return out
+
+    def ring(self) -> Tuple[int, int]:
+        """(device address, bytes) of the fused mode's ring of region slots; (0, 0) without a ring."""
+        out = ctypes.c_void_p()
+        nbytes = ctypes.c_int64()
+        rc = lib().t3_plan_ring(self._h, ctypes.byref(out), ctypes.byref(nbytes))
+        if rc != OK:
+            raise T3Error(rc, "t3_plan_ring")
+        return int(out.value or 0), int(nbytes.value)
 
     def gemm_rs_host(self, X_host: int, W_host: int, Y_host: int, stream: int = 0) -> None:
         """Host-pointer entry: H2D copies, the op, D2H copy, all on `stream`."""

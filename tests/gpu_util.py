@@ -22,9 +22,30 @@ def view_f32(ptr: int, shape) -> torch.Tensor:
 
 
 def poison_partials(plan) -> None:
-    """Fills the full partial buffers with NaN: a reducer that reads a tile before it landed shows up."""
+    """Fills the full partial buffers AND the fused mode's ring of region slots with NaN: a reducer that
+    reads a tile before it landed shows up.  (Not for update-in-place plans, whose accumulators must be zero.)"""
     ptr, nbytes = plan.partials()
     view_f32(ptr, (nbytes // 4,)).fill_(float("nan"))
+    rptr, rbytes = plan.ring()
+    if rptr:
+        view_f32(rptr, (rbytes // 4,)).fill_(float("nan"))
+
+
+BAND_BYTES = 4096
+BAND_PATTERN = 0xA5
+
+
+def banded(nbytes: int):
+    """A device buffer of nbytes with a 4 KiB guard band of a known byte pattern on each side.
+    Returns (whole uint8 tensor, byte offset of the payload)."""
+    whole = torch.full((nbytes + 2 * BAND_BYTES,), BAND_PATTERN, dtype=torch.uint8, device="cuda")
+    return whole, BAND_BYTES
+
+
+def bands_intact(whole: torch.Tensor) -> bool:
+    """True when both guard bands still hold the pattern (nothing was written outside the payload)."""
+    lo, hi = whole[:BAND_BYTES], whole[-BAND_BYTES:]
+    return bool((lo == BAND_PATTERN).all()) and bool((hi == BAND_PATTERN).all())
 
 
 def exported_partials(plan, R, M, N) -> np.ndarray:

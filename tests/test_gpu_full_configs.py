@@ -96,3 +96,41 @@ def test_backward_fc1_with_w_stored_k_by_n_and_16_bit_partials():
     assert torch.equal(Y.view(torch.int16), Y2.view(torch.int16))
     got = Y.float()[torch.from_numpy(rows).cuda()].cpu().numpy()
     assert oracle.max_rel_err(got, yref) <= 2e-2
+
+
+SWEEP = [w.name for w in wl.sweep_points()]
+# the four points with the largest partial workspace (4*R*M*N): also checked with fp32 output at 1e-4
+SWEEP_F32 = {w.name for w in sorted(wl.sweep_points(), key=lambda w: (w.R * w.M * w.N, w.K))[-4:]}
+
+
+@pytest.mark.parametrize("name", SWEEP)
+def test_sweep_point_row_sample(name):
+    """Every point of the shape sweep (R x M x H grid, K = 4H) at full size, default chunking, fused
+    mode - the launch configuration the bench's sweep times - on a row sample the oracle computes
+    exactly: every 64th row plus the first and last row of every chunk, all N columns, full K.  These
+    are the sizes at which element offsets pass 2^31 and the partial workspace reaches 8.6 GB."""
+    import torch
+    import gpu_util as gu
+    w = wl.by_name(name)
+    xb, wb = wl.make_inputs(w)
+    rows = wl.sample_rows(w.M, w.R, seed=w.resolved_seed(), stride=64)
+    yref = oracle.gemm_rs(xb, wb, w.R, rows=rows)
+    rms = float(np.sqrt(np.mean(yref ** 2)))
+    X, W = gu.upload(xb, wb)
+    del xb, wb
+    ridx = torch.from_numpy(rows).cuda()
+    dtypes = [t3.BF16_OUT_BF16] + ([t3.BF16_OUT_F32] if name in SWEEP_F32 else [])
+    for dtype in dtypes:
+        Y = gu.out_tensor(w.M, w.N, dtype)
+        with t3.Plan(w.M, w.N, w.K, w.R, dtype, None) as plan:
+            gu.poison_partials(plan)
+            gu.run_once(plan, t3.MODE_FUSED, X, W, Y)
+        assert bool(torch.isfinite(Y.float()).all())
+        err = oracle.max_rel_err(Y[ridx].float().cpu().numpy(), yref, rms=rms)
+        assert err <= TOL[dtype], (name, dtype, err)
+        # no missed slice anywhere: every chunk has the full sum's scale
+        chunk_rms = Y.float().reshape(w.R, w.chunk_rows, w.N).pow(2).mean(dim=(1, 2)).sqrt().cpu().numpy()
+        assert np.all(np.abs(chunk_rms / rms - 1.0) < 0.08), chunk_rms / rms
+        del Y
+    del X, W
+    torch.cuda.empty_cache()

@@ -33,7 +33,7 @@ def test_library_exports_every_declared_symbol():
         for name in sorted(declared):
             assert hasattr(L, name), f"{name} declared in t3.h but not exported by {os.path.basename(path)}"
     assert declared == set(t3.EXPORTS)
-    assert t3.version() == 100
+    assert t3.version() == 110
 
 
 def test_shape_validation_codes():

@@ -2,12 +2,14 @@
 service thread that cannot take cudaMalloc's device-wide synchronisation, a process whose device memory
 is all held by its own pool).  Its scratch is a static device array inside the library, so the test
 checks what such a caller relies on: same bits as the plan-based entry point, call after call, with the
-array reused (and its tracker words cleared) between calls.
+array reused (and its tracker words cleared) between calls; and, independently of the plan entry, the
+CPU oracle's values (bit for bit on exact-integer inputs, within the output tolerance on config 1).
 
 Collected last on purpose: a failure here cannot hide the other tests under `-x`."""
 import numpy as np
 import pytest
 
+import oracle
 from paper_2401_16677_b200 import build as t3build
 from paper_2401_16677_b200 import t3
 from paper_2401_16677_b200 import workloads as wl
@@ -52,6 +54,13 @@ def test_static_scratch_entry_matches_plan_entry_twice_in_a_row():
             torch.cuda.synchronize()
             got = gu.y_bits(Y)
             assert np.array_equal(got, want), f"{kind}: call {call} differs from t3_gemm_rs"
+            # and against the oracle itself, not only against the other entry point
+            yref = oracle.gemm_rs(xb, wb, R)
+            yf = Y.float().cpu().numpy().astype(np.float64)
+            if kind == "c1":
+                assert oracle.max_rel_err(yf, yref) <= 2e-2
+            else:
+                assert np.array_equal(yf, yref), f"{kind}: call {call} differs from the oracle"
 
 
 def test_static_scratch_entry_rejects_what_does_not_fit():
