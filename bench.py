@@ -43,7 +43,7 @@ NCU_TRAFFIC = {
     "C3b_megagpt_fc2": (1286.0e6, "profiles/t3_fused_kernel_C3b.md"),
 }
 CHUNK_ARGS = ("tile_n", "group_tiles", "reducer_ctas", "reducer_warps", "reduce_rows", "stages", "ring_slots", "cluster_ctas",
-              "partial_dtype", "order", "reduce", "split_k")
+              "partial_dtype", "order", "reduce", "split_k", "l2_hints")
 PER_CONFIG = ["C1_tiny", "C2_gpt2xl_fc2", "C3a_megagpt_attn_out", "C3b_megagpt_fc2", "C4_large_fc2:f32"]
 
 
@@ -247,7 +247,7 @@ def _interleaved(torch, t3, plan, X, W, Y, st, flush, rounds, per_round):
 
 
 def _overlap_figures(us, timeline):
-    """Exposed / hidden reduction from the per-round medians (Section 5.1.3's configurations: Sequential,
+    """Exposed / hidden reduction from the per-round medians (Section 5.3's configurations: Sequential,
     and the ideal overlap max(GEMM, RS))."""
     med = statistics.median
     f, q, g, r = (med(us[n]) for n in MODE_NAMES)
@@ -260,7 +260,7 @@ def _overlap_figures(us, timeline):
         "exposed_reduce_us": round(max(0.0, f - g), 2),
         "hidden_reduce_frac": round(1.0 - max(0.0, f - g) / r, 4),
         "hidden_reduce_frac_range": [round(min(per_round_hidden), 4), round(max(per_round_hidden), 4)],
-        # against the ideal overlap of Section 5.1.3: max(GEMM, reduction), no contention
+        # against the ideal overlap of Section 5.3: max(GEMM, reduction), no contention
         "ideal_overlap_us": round(max(g, r), 2),
         "exposed_vs_ideal_us": round(f - max(g, r), 2),
         # definition 2: inside the fused kernel itself - what is left after its last partial tile landed
@@ -318,6 +318,14 @@ def _per_config(torch, np, t3, wl, spec, st, flush, peaks, rounds, per_round):
     return entry
 
 
+def _workload(wl, args):
+    """The named workload, or (profiling aid) --shape M,N,K,R with the large-FC-2 value distributions."""
+    if args.shape:
+        M, N, K, R = (int(v) for v in args.shape.split(","))
+        return wl.Workload(f"shape_{M}x{N}x{K}_R{R}", M=M, N=N, K=K, R=R, x_dist="normal", w_dist="normal", w_std=0.01)
+    return wl.by_name(args.workload)
+
+
 def run_ours(args):
     import numpy as np
     import torch
@@ -346,7 +354,7 @@ def run_ours(args):
         dist.barrier()
     t3.lib()
 
-    w = wl.by_name(args.workload)
+    w = _workload(wl, args)
     dtype = t3.BF16_OUT_F32 if args.out == "f32" else t3.BF16_OUT_BF16
     xb, wb = wl.make_inputs(w)
     wnk = wl.w_nk(wb)
@@ -566,6 +574,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--shape", default="", help="profiling aid: M,N,K,R instead of a named workload (e.g. a configuration "
+                    "scaled down in M for an ncu capture)")
     ap.add_argument("--out", default="bf16", choices=["bf16", "f32"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--only", default=None, choices=["fused", "sequential", "gemm_only", "reduce_only"],

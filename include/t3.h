@@ -16,7 +16,7 @@
  * to a workspace, a counter per output tile counts landed partial tiles, and
  * the R-way sum of a tile (in the ring's order, Section 4.1) runs as soon as
  * its counter reaches its threshold, concurrently with the remaining GEMM
- * tiles.  The sequential baseline (Section 5.1.3, "Sequential": GEMM kernel,
+ * tiles.  The sequential baseline (Section 5.3, "Sequential": GEMM kernel,
  * then the collective's kernel) lives in the same library.
  *
  * All pointers named "device" are CUDA device pointers on the device that was
@@ -63,7 +63,7 @@ typedef enum {
 } t3_mode_t;
 
 /* Storage type of the per-slice partial tiles, i.e. what a device would put on the wire.  fp32 keeps
- * the 1e-4 tolerance of the fp32 output; bf16 follows Section 5.1.2's 16-bit setup: one extra
+ * the 1e-4 tolerance of the fp32 output; bf16 follows Section 5.2's 16-bit setup: one extra
  * round-to-nearest-even per slice, the ring sum itself stays fp32, half the reduction traffic. */
 typedef enum {
     T3_PARTIAL_F32 = 0,
@@ -110,6 +110,7 @@ typedef enum {
 
 /* debug_flags (host-made fault injection for the bounded-wait tests) */
 #define T3_DEBUG_INFLATE_EXPECTED 1   /* tracker thresholds +1: the trigger never fires, reducers time out */
+#define T3_DEBUG_NO_SPARE_REDUCERS 2  /* SMs without producer tiles stay idle instead of running reducers    */
 
 /*
  * How the output is tiled, tracked and reduced ("address-space configuration",
@@ -145,7 +146,12 @@ typedef struct {
                              /* reduce = T3_REDUCE_INPLACE when > 1; 0 = 1; at most 16 and at most    */
                              /* the slice's k-blocks.  For shapes with too few tiles to fill the GPU  */
                              /* (small M: the token-generation phase, Section 7.3).                  */
-    int32_t reserved[3];     /* must be zero                                                         */
+    int32_t l2_hints;        /* L2 eviction-priority hints, a bit mask; 0 = auto (the measured default), */
+                             /* -1 = none.  1: X tiles are fetched evict_last; 2: reducers read partial */
+                             /* tiles evict_first (their last use); 4 / 8: partial tiles are stored     */
+                             /* evict_last / evict_first; 16 / 32: W tiles are fetched evict_last /     */
+                             /* evict_first.  Performance only, never results.                          */
+    int32_t reserved[2];     /* must be zero                                                         */
 } t3_chunking_t;
 
 /* Geometry and cost model of a plan (all host-computed). */
@@ -271,7 +277,7 @@ int t3_gemm_rs_ex(t3_plan_t plan, const void *X, const void *W, void *Y,
 
 /* Same, in an explicit mode (the bench times FUSED, SEQUENTIAL, GEMM_ONLY and
  * REDUCE_ONLY on one plan so that all share one workspace and tile shape;
- * Section 5.1.3 configurations "Sequential" and the overlap comparison).
+ * Section 5.3 configurations "Sequential" and the overlap comparison).
  * X, W may be NULL for REDUCE_ONLY; Y may be NULL for GEMM_ONLY. */
 int t3_gemm_rs_mode(t3_plan_t plan, int32_t mode, const void *X, const void *W, void *Y,
                     void *stream);
@@ -391,7 +397,7 @@ int t3_plan_ring(t3_plan_t plan, void **ring /* host, receives device ptr */,
 
 /*
  * t3_plan_timeline - where the time of the plan's last FUSED call went
- * (Section 5.1.3 compares against an ideal overlap; this splits the fused
+ * (Section 5.3 compares against an ideal overlap; this splits the fused
  * kernel's own time the same way).  Every CTA records the GPU's global
  * nanosecond timer at four points; the call synchronises the plan's last
  * stream and reduces them:

@@ -104,6 +104,9 @@ struct alignas(64) KParams {
     int inplace;            // 1: update-in-place reduction (Section 4.3's analog): the epilogues add every slice's
                             // tile into ONE fp32 accumulator tile per region with L2 reductions; the tracker then
                             // gates only the final convert / store pass, which also clears the accumulator
+    int l2_hints;           // L2 eviction priorities: bit 0: X tiles fetched evict_last; bit 1: reducers read partial
+                            // tiles evict_first (their last use); bit 2 / 3: partial tiles stored evict_last /
+                            // evict_first; bit 4 / 5: W tiles fetched evict_last / evict_first
     EpiOps epi;             // element-wise work fused on the reduced chunk (Section 7.6)
     unsigned long long* trace;   // [grid][4] globaltimer: start, last tracker update, last reduced item, end; or NULL
 };
@@ -292,17 +295,30 @@ __device__ __forceinline__ void quad_exchange(float2& lo, float2& hi, int q) {
     if (up) lo = recv; else hi = recv;
 }
 
-// Reduces rows 8 * rowsel + [0, 8) of one 32 x 32 chunk: sums the R stored copies (slice d at
-// chunk + d * slice_stride) in ring order and writes the Y elements that exist.  Lane 4 g + q works on
-// row g of the group: its two float4 (jp = 0, 1) hold columns 8 j + 2 q + {0, 1}, j = 0..3.
-// row_base / col_base: global position of the chunk's element (0, 0); ncols_left: columns of the chunk
-// that exist (> 0, a multiple of 8).  All 32 lanes must call it (warp shuffles inside).
-// A lane keeps 2 x B 128-bit loads in flight.
+// The reduction of 32 x 32 chunks.  Lane 4 g + q works on row g of an 8-row group ("row group" rowsel of
+// the chunk): its two float4 (jp = 0, 1) of a stored copy hold columns 8 j + 2 q + {0, 1}, j = 0..3 (slice d's
+// copy of the chunk is at chunk + d * slice_stride).  row_base / col_base: global position of the chunk's
+// element (0, 0); ncols_left: columns of the chunk that exist (> 0, a multiple of 8).  All 32 lanes must
+// call (warp shuffles inside).
+// regroups one row's sums among the four lanes of the row and writes its eight neighbouring outputs
+__device__ __forceinline__ void finish_row(const float4 (&acc)[2], int q, void* Y, int M, int N, int out_f32, int row, int col_base,
+                                           int ncols_left, const EpiOps& eo) {
+    float2 a[4] = {make_float2(acc[0].x, acc[0].y), make_float2(acc[0].z, acc[0].w),
+                   make_float2(acc[1].x, acc[1].y), make_float2(acc[1].z, acc[1].w)};
+    quad_exchange<1>(a[0], a[1], q);
+    quad_exchange<1>(a[2], a[3], q);
+    quad_exchange<2>(a[0], a[2], q);
+    quad_exchange<2>(a[1], a[3], q);
+    if (row < M && 8 * q < ncols_left) store_y_8(Y, N, row, col_base + 8 * q, a, out_f32, eo);
+}
+
+// Sums the R stored copies of row group rowsel in ring order and writes the Y elements that exist; a lane
+// keeps 2 x B 128-bit loads in flight.
 template <int B>
 __device__ __forceinline__ void reduce_row_group(const float* __restrict__ chunk, size_t slice_stride, int rowsel,
                                                  void* Y, int M, int N, int R, int chunk_rows, int out_f32,
-                                                 int row_base, int col_base, int ncols_left, int lane,
-                                                 const EpiOps& eo) {
+                                                 int row_base, int col_base, int ncols_left, int lane, const EpiOps& eo,
+                                                 bool last_use, uint64_t pol_first) {
     const int g = lane >> 2, q = lane & 3;
     // float4 index of (rowsel, jp, lane): ((2 * rowsel + jp) * 32 + lane)
     const float* pos = chunk + (static_cast<size_t>(2 * rowsel) * 32 + lane) * 4;
@@ -317,8 +333,13 @@ __device__ __forceinline__ void reduce_row_group(const float* __restrict__ chunk
         for (int i = 0; i < B; ++i)
             if (s0 + i < R) {
                 const float* ps = pos + static_cast<size_t>(d) * slice_stride;
-                x[0][i] = ld_partial_v4(ps);
-                x[1][i] = ld_partial_v4(ps + 128);
+                if (last_use) {
+                    x[0][i] = ld_partial_v4_hint(ps, pol_first);
+                    x[1][i] = ld_partial_v4_hint(ps + 128, pol_first);
+                } else {
+                    x[0][i] = ld_partial_v4(ps);
+                    x[1][i] = ld_partial_v4(ps + 128);
+                }
                 d = d == 0 ? R - 1 : d - 1;
             }
 #pragma unroll
@@ -334,14 +355,7 @@ __device__ __forceinline__ void reduce_row_group(const float* __restrict__ chunk
                 }
             }
     }
-    // a[j]: columns 8 j + 2 q + {0, 1} of the row; after the transpose: columns 8 q + 2 j + {0, 1}
-    float2 a[4] = {make_float2(acc[0].x, acc[0].y), make_float2(acc[0].z, acc[0].w),
-                   make_float2(acc[1].x, acc[1].y), make_float2(acc[1].z, acc[1].w)};
-    quad_exchange<1>(a[0], a[1], q);
-    quad_exchange<1>(a[2], a[3], q);
-    quad_exchange<2>(a[0], a[2], q);
-    quad_exchange<2>(a[1], a[3], q);
-    if (row < M && 8 * q < ncols_left) store_y_8(Y, N, row, col_base + 8 * q, a, out_f32, eo);
+    finish_row(acc, q, Y, M, N, out_f32, row, col_base, ncols_left, eo);
 }
 
 // 16-bit partial tiles: the same reduction of one 8-row group; a lane reads its row's eight values of a
@@ -427,7 +441,7 @@ __device__ __noinline__ void finish_item_inplace(const float* __restrict__ chunk
 __device__ __forceinline__ void reduce_item(const void* __restrict__ chunk, size_t slice_stride, int partial_bf16,
                                             int row_in_block, int rows, void* Y, int M, int N, int R, int chunk_rows,
                                             int out_f32, int row_base, int col_base, int ncols_left, int lane,
-                                            const EpiOps& eo, int inplace) {
+                                            const EpiOps& eo, int inplace, int l2_hints = 0) {
     const int first = row_in_block >> 3;
     int end = (row_in_block + rows) >> 3;
     if (row_base + 8 * end > M) end = (M - row_base + 7) >> 3;     // the rest of the block is padding
@@ -440,10 +454,12 @@ __device__ __forceinline__ void reduce_item(const void* __restrict__ chunk, size
             reduce_row_group_bf16<8>(static_cast<const __nv_bfloat16*>(chunk), slice_stride, rowsel, Y, M, N, R, chunk_rows,
                                       out_f32, row_base, col_base, ncols_left, lane, eo);
     } else {
+        const bool last_use = (l2_hints & 2) != 0;
+        const uint64_t pol_first = l2_policy_evict_first();
 #pragma unroll 1
         for (int rowsel = first; rowsel < end; ++rowsel)
             reduce_row_group<8>(static_cast<const float*>(chunk), slice_stride, rowsel, Y, M, N, R, chunk_rows, out_f32,
-                                row_base, col_base, ncols_left, lane, eo);
+                                row_base, col_base, ncols_left, lane, eo, last_use, pol_first);
     }
 }
 
@@ -459,6 +475,19 @@ __device__ __forceinline__ void epi_store_frag(const uint32_t (&lo)[16], const u
         const uint32_t* src = rowsel < 2 ? lo : hi;
         asm volatile("st.global.v4.b32 [%0], {%1, %2, %3, %4};" ::"l"(p0 + i * 128), "r"(src[8 * jp + 2 * half]),
                      "r"(src[8 * jp + 2 * half + 1]), "r"(src[8 * jp + 4 + 2 * half]), "r"(src[8 * jp + 4 + 2 * half + 1])
+                     : "memory");
+    }
+}
+// the same with an L2 eviction-priority policy for the written lines
+__device__ __forceinline__ void epi_store_frag_hint(const uint32_t (&lo)[16], const uint32_t (&hi)[16], int lane,
+                                                    float* __restrict__ chunk, uint64_t policy) {
+    float* p0 = chunk + lane * 4;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int rowsel = i >> 1, jp = i & 1, half = rowsel & 1;
+        const uint32_t* src = rowsel < 2 ? lo : hi;
+        asm volatile("st.global.L2::cache_hint.v4.b32 [%0], {%1, %2, %3, %4}, %5;" ::"l"(p0 + i * 128), "r"(src[8 * jp + 2 * half]),
+                     "r"(src[8 * jp + 2 * half + 1]), "r"(src[8 * jp + 4 + 2 * half]), "r"(src[8 * jp + 4 + 2 * half + 1]), "l"(policy)
                      : "memory");
     }
 }
@@ -572,6 +601,9 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
             uint32_t ph = 0;
             bool ok = true;
             const uint32_t full0 = mapa_cluster(smem_u32(&bar_full[0]), lead);   // the pair leader's full barriers
+            const bool hint_x = (p.l2_hints & 1) != 0, hint_w = (p.l2_hints & 48) != 0;
+            const uint64_t pol_x = l2_policy_evict_last();
+            const uint64_t pol_w = (p.l2_hints & 16) ? l2_policy_evict_last() : l2_policy_evict_first();
             const int a_row_off = static_cast<int>(half) * BM;
             const int b_row_off = static_cast<int>(half) * (p.BN >> 1);
 #pragma unroll 1
@@ -594,7 +626,8 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                     if (elect_one_sync()) {
                         // a box is counted in full even where it is zero-filled
                         if (half == 0) mbar_arrive_expect_tx(smem_u32(&bar_full[s]), 2u * (p.a_bytes + p.b_bytes));
-                        tma_load_3d_pair(dst, &p.tmX, full, k0, r, a_row);
+                        if (hint_x) tma_load_3d_pair_hint(dst, &p.tmX, full, k0, r, a_row, pol_x);
+                        else tma_load_3d_pair(dst, &p.tmX, full, k0, r, a_row);
                         // W [N][K]: one box of BN/2 rows x 64 k.  W [K][N]: boxes of 64 k-rows x 64 columns
                         // (128 bytes), 8 KB apart in shared memory.
                         const int nbox = p.w_kn ? (p.BN >> 1) / 64 : 1;
@@ -607,6 +640,8 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                                 if (p.w_kn)
                                     for (int bx = 0; bx < nbox; ++bx)
                                         tma_load_3d_pair_shared(dstB + bx * 8192u, &p.tmW, full, b_row + bx * 64, k0, r, both);
+                                else if (hint_w)
+                                    tma_load_3d_pair_shared_hint(dstB, &p.tmW, full, k0, r, b_row, both, pol_w);
                                 else
                                     tma_load_3d_pair_shared(dstB, &p.tmW, full, k0, r, b_row, both);
                             }
@@ -615,6 +650,8 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                         if (p.w_kn) {
                             for (int bx = 0; bx < nbox; ++bx)
                                 tma_load_3d_pair(dstB + bx * 8192u, &p.tmW, full, b_row + bx * 64, k0, r);
+                        } else if (hint_w) {
+                            tma_load_3d_pair_hint(dstB, &p.tmW, full, k0, r, b_row, pol_w);
                         } else {
                             tma_load_3d_pair(dstB, &p.tmW, full, k0, r, b_row);
                         }
@@ -720,6 +757,8 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
         // Each warp owns 32 accumulator rows and walks them in 32-column chunks; the TMEM load of the
         // next chunk is in flight while the current one is transposed and stored.
         const int q = warp & 3;                                  // TMEM lane quarter this warp may read
+        const bool hint_st = (p.l2_hints & 12) != 0 && !p.partial_bf16 && !p.inplace;
+        const uint64_t pol_st = (p.l2_hints & 4) ? l2_policy_evict_last() : l2_policy_evict_first();
         const uint32_t tempty0 = mapa_cluster(smem_u32(&bar_tempty[0]), lead);   // the pair leader's
         int jl = 0, acc = 0;
         uint32_t acc_ph = 0;
@@ -805,6 +844,7 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                     if (lane == 0) mbar_arrive_cluster_relaxed(tempty0 + static_cast<uint32_t>(acc) * 8u);
                 }
                 if (p.inplace) epi_red_frag(alo, ahi, lane, dst + ci * FRAG_ELEMS);
+                else if (hint_st) epi_store_frag_hint(alo, ahi, lane, dst + ci * FRAG_ELEMS, pol_st);
                 else if (p.partial_bf16) epi_store_frag_bf16(alo, ahi, lane, dst16 + ci * FRAG_ELEMS);
                 else epi_store_frag(alo, ahi, lane, dst + ci * FRAG_ELEMS);
                 if (ci + 1 < nchunks) {
@@ -818,6 +858,7 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                         if (lane == 0) mbar_arrive_cluster_relaxed(tempty0 + static_cast<uint32_t>(acc) * 8u);
                     }
                     if (p.inplace) epi_red_frag(blo, bhi, lane, dst + (ci + 1) * FRAG_ELEMS);
+                    else if (hint_st) epi_store_frag_hint(blo, bhi, lane, dst + (ci + 1) * FRAG_ELEMS, pol_st);
                     else if (p.partial_bf16) epi_store_frag_bf16(blo, bhi, lane, dst16 + (ci + 1) * FRAG_ELEMS);
                     else epi_store_frag(blo, bhi, lane, dst + (ci + 1) * FRAG_ELEMS);
                 }
@@ -862,7 +903,7 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                                         ? static_cast<const void*>(reinterpret_cast<const __nv_bfloat16*>(p.partials) + chunk_off)
                                         : static_cast<const void*>(p.partials + chunk_off);
                 reduce_item(chunk, static_cast<size_t>(p.tile_elems), p.partial_bf16, rib, p.sched.reduce_rows, p.Y, p.M, p.N,
-                            p.R, p.chunk_rows, p.out_f32, row_base, col_base, ncols_left, lane, p.epi, p.inplace);
+                            p.R, p.chunk_rows, p.out_f32, row_base, col_base, ncols_left, lane, p.epi, p.inplace, p.l2_hints);
                 if (p.ring_slots > 0) {
                     // every lane's loads of this item have returned (their values were used above)
                     __syncwarp();

@@ -50,7 +50,7 @@ constexpr int EPI_WARPS = 4;
 //   col in chunk = 16 * jp + 8 * (e >> 1) + 2 * q + (e & 1)   (jp 0..1, q 0..3, e 0..3)
 // A float4 therefore holds two pairs of neighbouring columns of one row; the reducer regroups the
 // sums among the four lanes of a row before it writes Y.
-// With 16-bit partial tiles (the "wire" type of Section 5.1.2) a chunk is 1024 bf16 and a lane's eight
+// With 16-bit partial tiles (the "wire" type of Section 5.2) a chunk is 1024 bf16 and a lane's eight
 // values of one row (jp = 0 and 1) are stored together as 16 bytes:
 //   bf16 index = ((rowsel * 32 + lane) * 8 + jp * 4 + e
 // so a chunk is written with four and read with four 128-bit accesses per lane.

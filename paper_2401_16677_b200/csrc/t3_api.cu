@@ -52,6 +52,7 @@ struct Geometry {
     t3::Sched sched;
     int k_align;              // k-blocks may start on 128-byte lines (row pitch is a multiple of 128 bytes)
     uint32_t a_bytes, b_bytes, stage_bytes;
+    int spare_reducers;       // reducer-only CTAs added on SMs that have no producer tiles (part of info.reducer_ctas)
 };
 
 int pick_tile_n(int64_t N, int step) {
@@ -88,7 +89,12 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
     t3_chunking_t c;
     std::memset(&c, 0, sizeof c);
     if (in) c = *in;
-    if (c.reserved[0] != 0 || c.reserved[1] != 0 || c.reserved[2] != 0) return T3_ERR_INVALID_ARG;
+    if (c.reserved[0] != 0 || c.reserved[1] != 0) return T3_ERR_INVALID_ARG;
+    if (c.l2_hints < -1 || c.l2_hints > 63 || (c.l2_hints > 0 && ((c.l2_hints & 12) == 12 || (c.l2_hints & 48) == 48))) return T3_ERR_INVALID_ARG;
+    // measured (interleaved, four configurations): X tiles kept (they are reused by every column tile of a schedule
+    // group) and partial tiles released by the reducers' reads are worth 2-6 %; W evict_first pays only where W
+    // has no reuse in L2 (the largest shape: 28 % less DRAM read traffic, same time), so it stays an option
+    if (c.l2_hints == 0) c.l2_hints = 3;
     if (c.reduce != T3_REDUCE_RING && c.reduce != T3_REDUCE_INPLACE) return T3_ERR_INVALID_ARG;
     if (c.order != T3_ORDER_GROUPED && c.order != T3_ORDER_STAGGERED) return T3_ERR_INVALID_ARG;
     if (c.w_layout != T3_W_NK && c.w_layout != T3_W_KN) return T3_ERR_INVALID_ARG;
@@ -171,6 +177,7 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
     if (c.stages < 2 || c.stages > t3::MAX_STAGES || c.stages > max_stages) return T3_ERR_INVALID_ARG;
 
     g.cfg = c;
+    g.spare_reducers = 0;
     g.a_bytes = a_bytes;
     g.b_bytes = b_bytes;
     g.stage_bytes = stage_bytes;
@@ -211,7 +218,16 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
     o.grid = grid;
     o.reducer_ctas = c.reducer_ctas;
     o.gemm_ctas = grid - c.reducer_ctas;
-    if (o.gemm_ctas > t3::CTA_PAIR * o.n_jobs) o.gemm_ctas = t3::CTA_PAIR * o.n_jobs;
+    if (o.gemm_ctas > t3::CTA_PAIR * o.n_jobs) {
+        // fewer producer tiles than CTA pairs (small M: Section 7.3's generation phase, or a tiny problem):
+        // the SMs left over run reducers only instead of idling, which shortens the reduction that starts
+        // when the one wave of tiles lands
+        o.gemm_ctas = t3::CTA_PAIR * o.n_jobs;
+        if (c.mode == T3_MODE_FUSED && c.reducer_ctas == 0 && !(c.debug_flags & T3_DEBUG_NO_SPARE_REDUCERS)) {
+            g.spare_reducers = (grid - o.gemm_ctas) / cl * cl;
+            o.reducer_ctas = g.spare_reducers;
+        }
+    }
     o.grid = o.gemm_ctas + o.reducer_ctas;
     o.reducer_warps = c.reducer_warps;
     o.reduce_rows = c.reduce_rows;
@@ -538,6 +554,7 @@ void fill_params(t3_plan_t pl, const Geometry& g, void* Y, bool with_reduce, con
     kp.timeout_ns = static_cast<unsigned long long>(g.cfg.timeout_ms) * 1000000ull;
     kp.inplace = g.cfg.reduce == T3_REDUCE_INPLACE;
     kp.split_k = g.info.split_k;
+    kp.l2_hints = g.cfg.l2_hints > 0 ? g.cfg.l2_hints : 0;
     kp.epi = epi;
     kp.trace = (with_reduce && g.info.grid <= pl->trace_ctas) ? pl->trace : nullptr;
 }
@@ -576,6 +593,15 @@ int fit_to_device(Geometry& g, int smem_optin) {
     const int cl = oi.cluster_ctas;
     const int max_clusters = prepare_kernel(cl, oi.grid, smem_optin);
     if (max_clusters < 1) return T3_ERR_CUDA;
+    if (oi.grid > cl * max_clusters && g.spare_reducers > 0) {
+        // the reducer-only CTAs that were added to fill idle SMs go first
+        int cut = oi.grid - cl * max_clusters;
+        cut = (cut + cl - 1) / cl * cl;
+        if (cut > g.spare_reducers) cut = g.spare_reducers;
+        g.spare_reducers -= cut;
+        oi.reducer_ctas -= cut;
+        oi.grid -= cut;
+    }
     if (oi.grid > cl * max_clusters) {
         const int new_grid = cl * max_clusters;
         if (oi.reducer_ctas >= new_grid) return T3_ERR_UNSUPPORTED;
@@ -1065,6 +1091,7 @@ int t3_gemm_rs_static(int64_t M, int64_t N, int64_t K, int32_t R, t3_dtype_t dty
     ch.mode = T3_MODE_FUSED;
     ch.ring_slots = -1;                       // partial tiles in full buffers, inside the static array
     ch.cluster_ctas = t3::CTA_PAIR;
+    ch.l2_hints = -1;
     Geometry g;                               // on the stack: no heap either
     rc = resolve_geometry(M, N, K, R, static_cast<int>(dtype), &ch, st->sm_count, g);
     if (rc != T3_OK) return fail(rc);

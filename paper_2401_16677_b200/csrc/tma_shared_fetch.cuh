@@ -19,4 +19,15 @@ __device__ __forceinline__ void tma_load_3d_pair_shared(uint32_t dst, const void
         : "memory");
 }
 
+// The same with an L2 eviction-priority policy for the fetched lines.
+__device__ __forceinline__ void tma_load_3d_pair_shared_hint(uint32_t dst, const void* tmap, uint32_t cluster_bar, int c0,
+                                                             int c1, int c2, uint16_t cta_mask, uint64_t policy) {
+    asm volatile(
+        "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.multicast::cluster"
+        ".L2::cache_hint [%0], [%1, {%3, %4, %5}], [%2], %6, %7;"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(tmap)), "r"(cluster_bar), "r"(c0), "r"(c1), "r"(c2), "h"(cta_mask),
+          "l"(policy)
+        : "memory");
+}
+
 }  // namespace t3

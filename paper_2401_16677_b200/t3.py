@@ -76,7 +76,8 @@ class Chunking(ctypes.Structure):
         ("stages", ctypes.c_int32), ("timeout_ms", ctypes.c_int32), ("debug_flags", ctypes.c_int32),
         ("max_ctas", ctypes.c_int32), ("ring_slots", ctypes.c_int32), ("cluster_ctas", ctypes.c_int32),
         ("partial_dtype", ctypes.c_int32), ("w_layout", ctypes.c_int32), ("order", ctypes.c_int32),
-        ("reduce", ctypes.c_int32), ("split_k", ctypes.c_int32), ("reserved", ctypes.c_int32 * 3),
+        ("reduce", ctypes.c_int32), ("split_k", ctypes.c_int32), ("l2_hints", ctypes.c_int32),
+        ("reserved", ctypes.c_int32 * 2),
     ]
 
 

@@ -6,7 +6,7 @@ neither the CUDA binding nor the CPU oracle, and is the one piece both sides
 share: tests and the bench feed the very same bf16 bit patterns to each.
 
 Shapes follow the paper's sliced sublayers (Section 2.4: a weight sliced
-along its dot-product dimension over the tensor-parallel group; Section 5.1.2
+along its dot-product dimension over the tensor-parallel group; Section 5.2
 and the model table: token counts of 8K-16K, TP degrees 8/16).  Value
 distributions are synthetic stand-ins for trained activations and weights.
 
@@ -78,7 +78,7 @@ C4 = Workload("C4_large_fc2", M=4096, N=8192, K=32768, R=16,
 CONFIGS: Dict[str, Workload] = {w.name: w for w in (C1, C2, C3A, C3B, C4)}
 
 # Backward-pass sublayers that need the same sliced GEMM + all-reduce (Section 2.4 and the sublayer
-# list of Section 5.1.2): the input-gradient GEMMs of the input projection (K = 3H) and of FC-1
+# list of Section 5.2): the input-gradient GEMMs of the input projection (K = 3H) and of FC-1
 # (K = 4H, the same shape as the forward FC-2), at the Mega-GPT-like width.  Incoming gradients are
 # drawn small and zero-mean like activations' gradients.
 X_BWD_IP = Workload("X_megagpt_bwd_ip", M=4096, N=3072, K=9216, R=8,

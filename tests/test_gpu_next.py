@@ -405,3 +405,4 @@ def test_guard_bands_around_y_and_export_buffer(M, N, K, R, dtype):
             got = _to_f64(Y)
             ref = want if dtype == t3.BF16_OUT_F32 else wl.bf16_bits_to_f64(wl.f32_to_bf16_bits(want.astype(np.float32)))
             assert np.array_equal(got, ref)
+
