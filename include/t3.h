@@ -116,6 +116,11 @@ typedef enum {
  * How the output is tiled, tracked and reduced ("address-space configuration",
  * Section 4.4: what to track, at which granularity, trigger condition).
  * Zero in any field selects the default.  NULL selects all defaults.
+ * For the fields tile_n, group_tiles, reducer_ctas, reducer_warps, reduce_rows,
+ * ring_slots, cluster_ctas, timeout_ms and l2_hints a zero is first replaced
+ * by the integer in the environment variable T3_<FIELD NAME IN CAPITALS>
+ * (T3_RING_SLOTS, T3_TIMEOUT_MS, ...) when that is set; values a shape does
+ * not admit give the usual error code.
  */
 typedef struct {
     int32_t mode;            /* t3_mode_t used by t3_gemm_rs                                         */
@@ -344,11 +349,13 @@ int t3_gemm_rs_static(int64_t M, int64_t N, int64_t K, int32_t R, t3_dtype_t dty
  * from the producer kernel's behaviour while it runs alone in the first
  * stage; here a short trial on the real operands decides how the reduction
  * shares the GPU with the GEMM).  Runs the op a few times per candidate on
- * `stream`, timing with CUDA events, and keeps the fastest of
+ * `stream`, timing with CUDA events, each timed call after a rewrite of the
+ * plan's partial buffers (up to 512 MiB) that sweeps the L2, and keeps the
+ * fastest of
  *   { fused with the L2 ring, fused with full partial buffers, sequential }
  *   x reduce_rows { 16, 32 } x cluster_ctas { 2, 4 where available } x group height { g, g/2 }
  * that fit the plan's existing workspace (nothing is allocated).  A candidate
- * replaces the current configuration only if it is at least 2 % faster.  All
+ * replaces the current configuration only if it is at least 3 % faster.  All
  * candidates produce the same bits, so tuning never changes a result
  * (T3_REDUCE_INPLACE plans: within its stated non-determinism).
  * Synchronous: returns after the trials; Y holds a valid result.  out (host,

@@ -55,6 +55,17 @@ struct Geometry {
     int spare_reducers;       // reducer-only CTAs added on SMs that have no producer tiles (part of info.reducer_ctas)
 };
 
+// A field the caller left at 0 (= automatic) takes its value from the environment variable `name` when that
+// is set to an integer: a way to steer the automatic choices of code that passes NULL for the chunking.
+void env_default(int32_t& field, const char* name) {
+    if (field != 0) return;
+    const char* v = std::getenv(name);
+    if (!v || !*v) return;
+    char* end = nullptr;
+    const long x = std::strtol(v, &end, 10);
+    if (end != v && *end == 0 && x >= -1 && x <= 1 << 20) field = static_cast<int32_t>(x);
+}
+
 int pick_tile_n(int64_t N, int step) {
     // multiple of `step` in [128,256] with the least padded width; ties -> widest
     int best = 256;
@@ -90,11 +101,17 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
     std::memset(&c, 0, sizeof c);
     if (in) c = *in;
     if (c.reserved[0] != 0 || c.reserved[1] != 0) return T3_ERR_INVALID_ARG;
+    env_default(c.tile_n, "T3_TILE_N");
+    env_default(c.group_tiles, "T3_GROUP_TILES");
+    env_default(c.reducer_ctas, "T3_REDUCER_CTAS");
+    env_default(c.reducer_warps, "T3_REDUCER_WARPS");
+    env_default(c.reduce_rows, "T3_REDUCE_ROWS");
+    env_default(c.ring_slots, "T3_RING_SLOTS");
+    env_default(c.cluster_ctas, "T3_CLUSTER_CTAS");
+    env_default(c.timeout_ms, "T3_TIMEOUT_MS");
+    env_default(c.l2_hints, "T3_L2_HINTS");
     if (c.l2_hints < -1 || c.l2_hints > 63 || (c.l2_hints > 0 && ((c.l2_hints & 12) == 12 || (c.l2_hints & 48) == 48))) return T3_ERR_INVALID_ARG;
-    // measured (interleaved, four configurations): X tiles kept (they are reused by every column tile of a schedule
-    // group) and partial tiles released by the reducers' reads are worth 2-6 %; W evict_first pays only where W
-    // has no reuse in L2 (the largest shape: 28 % less DRAM read traffic, same time), so it stays an option
-    if (c.l2_hints == 0) c.l2_hints = 3;
+    const bool l2_auto = c.l2_hints == 0;      // resolved once the cluster size is known
     if (c.reduce != T3_REDUCE_RING && c.reduce != T3_REDUCE_INPLACE) return T3_ERR_INVALID_ARG;
     if (c.order != T3_ORDER_GROUPED && c.order != T3_ORDER_STAGGERED) return T3_ERR_INVALID_ARG;
     if (c.w_layout != T3_W_NK && c.w_layout != T3_W_KN) return T3_ERR_INVALID_ARG;
@@ -150,6 +167,14 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
         if (c.cluster_ctas == 0) c.cluster_ctas = (can4 && (flops >= 1e12 || R >= 16)) ? 4 : 2;
     }
     const int cl = c.cluster_ctas;
+    // L2 eviction priorities, measured (interleaved timings and DRAM-traffic captures): X tiles kept (a schedule
+    // group's X rows are reused by every column tile) and partial tiles released by the reducers' reads are
+    // worth 2-6 % everywhere.  In clusters of four both row tiles that use a W tile sit in the same cluster, so
+    // W lines have no further use once fetched: marking them evict_first, and the partial tiles evict_last
+    // until they are read, lets the ring of region slots survive in L2 (large FC-2 shape scaled to 1 024 rows:
+    // 2.37 -> 1.37 GB of DRAM traffic per launch).  That holds for two-tile groups only; taller groups (and
+    // pairs) reuse a W tile across the group's row tiles, and there W evict_first costs 5-20 %.
+    if (l2_auto) c.l2_hints = (cl == 4 && c.group_tiles == 2) ? 39 : 3;
     int grid = sm_count / cl * cl;                 // whole clusters
     if (c.max_ctas > 0 && c.max_ctas < grid) grid = c.max_ctas / cl * cl;
     if (grid < cl) return T3_ERR_INVALID_ARG;
@@ -249,8 +274,13 @@ int resolve_geometry(int64_t M, int64_t N, int64_t K, int32_t R, int dtype, cons
         const int pairs = (grid - c.reducer_ctas) / t3::CTA_PAIR;
         int64_t want = c.ring_slots;
         if (want == 0) {
-            want = (64ll << 20) / slot_bytes;      // about half of the 126 MB L2
-            const int64_t in_flight = (2ll * pairs + Rv - 1) / Rv + 2ll * c.group_tiles;
+            // about half of the 126 MB L2; a third where W streams through with no reuse (clusters of four on
+            // two-tile groups): the ring then stays resident beside the group's X rows (measured on the large
+            // FC-2 shape: 16 slots of 4 MB spill to DRAM entirely, 8-10 stay, 6 stall the producers)
+            const int64_t target = (cl == 4 && c.group_tiles == 2) ? (40ll << 20) : (64ll << 20);
+            want = target / slot_bytes;
+            // regions in production (one per R jobs in flight) plus two groups' worth waiting for reducers
+            const int64_t in_flight = (pairs + Rv - 1) / Rv + 2ll * c.group_tiles + 1;
             if (want < in_flight) want = in_flight;
         }
         if (want < 0) want = 0;                                   // -1: full partial buffers in fused mode too
@@ -1186,6 +1216,9 @@ int t3_plan_tune(t3_plan_t pl, const void* X, const void* W, void* Y, void* stre
         return fail(T3_ERR_CUDA);
     }
     constexpr int MAX_CAND = 48, TIMED = 5;
+    // the plan's own full partial buffers double as the buffer whose rewrite sweeps the L2 between timed
+    // calls: every mode rewrites them before reading them (update in place: they hold zeros between calls)
+    const size_t flush_bytes = std::min(static_cast<size_t>(cur.partial_bytes), static_cast<size_t>(512) << 20);
     Geometry best = cur;
     float best_us = 0.f, cur_us = 0.f;
     int n = 0, chosen = 0;
@@ -1225,11 +1258,14 @@ int t3_plan_tune(t3_plan_t pl, const void* X, const void* W, void* Y, void* stre
                     }
                     if (g.info.tile_n != o.tile_n || g.partial_bytes != cur.partial_bytes) continue;
                     if (fit_to_device(g, pl->smem_optin) != T3_OK) continue;
-                    // one untimed call, then TIMED timed ones
+                    // one untimed call, then TIMED timed ones, each after the L2 has been swept (a sublayer's
+                    // operands are cold when it runs inside a model: other layers' weights have passed through
+                    // the cache since its last call)
                     float us[TIMED];
                     bool ok = run_mode(pl, g, c.mode, Y, st, no_epi) == T3_OK;
                     for (int t = 0; ok && t < TIMED; ++t) {
-                        ok = cudaEventRecord(e0, st) == cudaSuccess && run_mode(pl, g, c.mode, Y, st, no_epi) == T3_OK &&
+                        ok = cudaMemsetAsync(pl->partials, 0, flush_bytes, st) == cudaSuccess &&
+                             cudaEventRecord(e0, st) == cudaSuccess && run_mode(pl, g, c.mode, Y, st, no_epi) == T3_OK &&
                              cudaEventRecord(e1, st) == cudaSuccess && cudaEventSynchronize(e1) == cudaSuccess;
                         float ms = 0.f;
                         ok = ok && cudaEventElapsedTime(&ms, e0, e1) == cudaSuccess;
@@ -1257,8 +1293,8 @@ int t3_plan_tune(t3_plan_t pl, const void* X, const void* W, void* Y, void* stre
     cudaEventDestroy(e0);
     cudaEventDestroy(e1);
     if (n == 0) return fail(T3_ERR_CUDA);
-    // keep the current configuration unless the best candidate is at least 2 % faster
-    if (chosen != 0 && best_us > 0.98f * cur_us) {
+    // keep the current configuration unless the best candidate is at least 3 % faster
+    if (chosen != 0 && best_us > 0.97f * cur_us) {
         best = cur;
         chosen = 0;
     }

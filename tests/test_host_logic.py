@@ -278,3 +278,16 @@ def test_multicast_variant_is_never_chosen_in_a_multi_process_launch():
                                    "from paper_2401_16677_b200 import t3; print(t3.LIB_PATH); "
                                    "print(t3.shared_fetch_available())"], cwd=ROOT, env=env, text=True).split()
     assert out[0] == portable and out[1] == "False"
+
+
+def test_environment_overrides_fill_only_fields_left_at_zero():
+    import subprocess
+    code = ("from paper_2401_16677_b200 import t3; "
+            "g = t3.geometry(4096, 3072, 12288, 8); "
+            "h = t3.geometry(4096, 3072, 12288, 8, chunk=t3.chunking(group_tiles=2, ring_slots=20)); "
+            "print(g.group_tiles, g.ring_slots, g.reduce_rows, h.group_tiles, h.ring_slots)")
+    env = dict(os.environ, T3_GROUP_TILES="4", T3_RING_SLOTS="24", T3_REDUCE_ROWS="16", T3_TIMEOUT_MS="junk")
+    out = subprocess.check_output([sys.executable, "-c", code], cwd=ROOT, env=env, text=True).split()
+    assert out == ["4", "24", "16", "2", "20"]
+    base = t3.geometry(4096, 3072, 12288, 8)
+    assert (base.group_tiles, base.reduce_rows) == (8, 32)
