@@ -40,9 +40,9 @@ L2_FLUSH_BYTES = 512 << 20
 # under profiles/ that holds the capture's command and figures.  Absent: no capture for that workload.
 NCU_TRAFFIC = {
     "C2_gpt2xl_fc2": (727.6e6, "profiles/t3_fused_kernel_C2.md"),
-    "C3b_megagpt_fc2": (1350.3e6, "profiles/t3_fused_kernel_C3b.md"),
-    # captured on the same shape scaled to M = 1 024 (1.372 GB per launch); traffic is proportional to M there
-    "C4_large_fc2": (4 * 1.372e9, "profiles/t3_fused_kernel_C4_scaled.md, x4 from the M = 1 024 capture"),
+    "C3b_megagpt_fc2": (1303.0e6, "profiles/t3_fused_kernel_C3b.md"),
+    # captured on the same shape scaled to M = 1 024 (1.609 GB per launch); traffic is proportional to M there
+    "C4_large_fc2": (4 * 1.609e9, "profiles/t3_fused_kernel_C4_scaled.md, x4 from the M = 1 024 capture"),
 }
 CHUNK_ARGS = ("tile_n", "group_tiles", "reducer_ctas", "reducer_warps", "reduce_rows", "stages", "ring_slots", "cluster_ctas",
               "partial_dtype", "order", "reduce", "split_k", "l2_hints")

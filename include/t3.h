@@ -232,12 +232,15 @@ t3_plan_t t3_plan(int64_t M, int64_t N, int64_t K, int32_t R, t3_dtype_t dtype,
  * One call in flight per plan.  The kernel is persistent (one CTA per SM, all
  * CTA pairs must be resident together because reducers wait on tiles other
  * pairs produce), so two t3 kernels must never share a GPU.  The library
- * sees to that itself: every launch made through a plan first waits, on its
- * stream, for an event recorded after the previous t3 launch on the same
- * device (whatever plan or stream that was), without blocking the host;
- * calls from several streams or host threads therefore run one after the
- * other on the GPU.  (Not inside a stream capture: a captured call is ordered
- * by its graph alone.  Not for t3_gemm_rs_static, which creates nothing.)
+ * sees to that itself: a call made on a different stream than the previous
+ * t3 launch on the same device (whatever plan that was) first makes its
+ * stream wait, on the GPU and without blocking the host, for the work
+ * enqueued so far on that previous stream; calls that follow each other on
+ * one stream pay nothing.  Calls from several streams or host threads
+ * therefore run one after the other on the GPU.  (Not inside a stream
+ * capture: a captured call is ordered by its graph alone.  Not for
+ * t3_gemm_rs_static, which creates nothing.  A stream must outlive the next
+ * t3 call made on another stream.)
  * The plan must be used with the device it was made on current
  * (T3_ERR_DEVICE otherwise).  Host-detectable errors return a negative code
  * and enqueue nothing; device-side timeouts are reported by t3_plan_status;
@@ -355,7 +358,8 @@ int t3_gemm_rs_static(int64_t M, int64_t N, int64_t K, int32_t R, t3_dtype_t dty
  *   { fused with the L2 ring, fused with full partial buffers, sequential }
  *   x reduce_rows { 16, 32 } x cluster_ctas { 2, 4 where available } x group height { g, g/2 }
  * that fit the plan's existing workspace (nothing is allocated).  A candidate
- * replaces the current configuration only if it is at least 3 % faster.  All
+ * replaces the current configuration only if it is at least 3 % faster (5 %
+ * if it is the sequential mode).  All
  * candidates produce the same bits, so tuning never changes a result
  * (T3_REDUCE_INPLACE plans: within its stated non-determinism).
  * Synchronous: returns after the trials; Y holds a valid result.  out (host,

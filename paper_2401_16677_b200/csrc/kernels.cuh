@@ -233,9 +233,8 @@ __device__ __forceinline__ void load_8(const void* base, size_t idx, int is_f32,
     }
 }
 
-// The element-wise tail of Section 7.6 on one row's eight neighbouring sums (columns col .. col + 7).  A real
-// call, not inlined: its registers are then needed only while it runs, not across the reducers' load rounds.
-__device__ __noinline__ void apply_epi_8(const EpiOps& eo, int N, int row, int col, float (&v)[8]) {
+// The element-wise tail of Section 7.6 on one row's eight neighbouring sums (columns col .. col + 7).
+__device__ __forceinline__ void apply_epi_8(const EpiOps& eo, int N, int row, int col, float (&v)[8]) {
     const size_t off = static_cast<size_t>(row) * static_cast<size_t>(N) + col;
     // issue the per-element loads first, then the (cached) bias
     uint2 km = make_uint2(0x01010101u, 0x01010101u);
@@ -263,11 +262,12 @@ __device__ __noinline__ void apply_epi_8(const EpiOps& eo, int N, int row, int c
 
 // One row's eight neighbouring outputs (columns col .. col + 7): the element-wise tail, if any, then one
 // rounding to the output type.
+template <bool EPI>
 __device__ __forceinline__ void store_y_8(void* Y, int N, int row, int col, const float2 (&a)[4], int out_f32,
                                           const EpiOps& eo) {
     const size_t off = static_cast<size_t>(row) * static_cast<size_t>(N) + col;
     float v[8] = {a[0].x, a[0].y, a[1].x, a[1].y, a[2].x, a[2].y, a[3].x, a[3].y};
-    if (eo.any) apply_epi_8(eo, N, row, col, v);
+    if (EPI && eo.any) apply_epi_8(eo, N, row, col, v);
     if (out_f32) {
         float4* dst = reinterpret_cast<float4*>(static_cast<float*>(Y) + off);
         dst[0] = make_float4(v[0], v[1], v[2], v[3]);
@@ -301,6 +301,7 @@ __device__ __forceinline__ void quad_exchange(float2& lo, float2& hi, int q) {
 // element (0, 0); ncols_left: columns of the chunk that exist (> 0, a multiple of 8).  All 32 lanes must
 // call (warp shuffles inside).
 // regroups one row's sums among the four lanes of the row and writes its eight neighbouring outputs
+template <bool EPI>
 __device__ __forceinline__ void finish_row(const float4 (&acc)[2], int q, void* Y, int M, int N, int out_f32, int row, int col_base,
                                            int ncols_left, const EpiOps& eo) {
     float2 a[4] = {make_float2(acc[0].x, acc[0].y), make_float2(acc[0].z, acc[0].w),
@@ -309,12 +310,12 @@ __device__ __forceinline__ void finish_row(const float4 (&acc)[2], int q, void* 
     quad_exchange<1>(a[2], a[3], q);
     quad_exchange<2>(a[0], a[2], q);
     quad_exchange<2>(a[1], a[3], q);
-    if (row < M && 8 * q < ncols_left) store_y_8(Y, N, row, col_base + 8 * q, a, out_f32, eo);
+    if (row < M && 8 * q < ncols_left) store_y_8<EPI>(Y, N, row, col_base + 8 * q, a, out_f32, eo);
 }
 
 // Sums the R stored copies of row group rowsel in ring order and writes the Y elements that exist; a lane
 // keeps 2 x B 128-bit loads in flight.
-template <int B>
+template <int B, bool EPI>
 __device__ __forceinline__ void reduce_row_group(const float* __restrict__ chunk, size_t slice_stride, int rowsel,
                                                  void* Y, int M, int N, int R, int chunk_rows, int out_f32,
                                                  int row_base, int col_base, int ncols_left, int lane, const EpiOps& eo,
@@ -355,7 +356,7 @@ __device__ __forceinline__ void reduce_row_group(const float* __restrict__ chunk
                 }
             }
     }
-    finish_row(acc, q, Y, M, N, out_f32, row, col_base, ncols_left, eo);
+    finish_row<EPI>(acc, q, Y, M, N, out_f32, row, col_base, ncols_left, eo);
 }
 
 // 16-bit partial tiles: the same reduction of one 8-row group; a lane reads its row's eight values of a
@@ -400,13 +401,13 @@ __device__ __forceinline__ void reduce_row_group_bf16(const __nv_bfloat16* __res
     quad_exchange<1>(a[2], a[3], q);
     quad_exchange<2>(a[0], a[2], q);
     quad_exchange<2>(a[1], a[3], q);
-    if (row < M && 8 * q < ncols_left) store_y_8(Y, N, row, col_base + 8 * q, a, out_f32, eo);
+    if (row < M && 8 * q < ncols_left) store_y_8<true>(Y, N, row, col_base + 8 * q, a, out_f32, eo);
 }
 
 // Update-in-place mode: the chunk holds the finished sums.  All row groups [first, end) of the item (at
 // most four) are read with their loads in flight together, cleared for the next call, regrouped among
 // the four lanes of a row and written to Y.
-__device__ __noinline__ void finish_item_inplace(const float* __restrict__ chunk, int first, int end, void* Y, int M, int N,
+__device__ __forceinline__ void finish_item_inplace(const float* __restrict__ chunk, int first, int end, void* Y, int M, int N,
                                                     int out_f32, int row_base, int col_base, int ncols_left, int lane,
                                                     const EpiOps& eo) {
     const int g = lane >> 2, q = lane & 3;
@@ -431,24 +432,37 @@ __device__ __noinline__ void finish_item_inplace(const float* __restrict__ chunk
             quad_exchange<2>(a[0], a[2], q);
             quad_exchange<2>(a[1], a[3], q);
             const int row = row_base + 8 * (first + i) + g;
-            if (row < M && 8 * q < ncols_left) store_y_8(Y, N, row, col_base + 8 * q, a, out_f32, eo);
+            if (row < M && 8 * q < ncols_left) store_y_8<true>(Y, N, row, col_base + 8 * q, a, out_f32, eo);
         }
 }
 
+// How a region's stored tiles become Y: a compile-time property of the kernels, so that each instantiation
+// holds exactly one variant of the reducers' inner loop and no call.  (Several inlined variants in one
+// branch made ptxas spill hundreds of bytes; real calls inside the row-group loop cost the reducers 5-6 %
+// on the reduction-heavy shapes because registers then follow the calling convention across the load rounds.)
+enum RMode {
+    RMODE_RING = 0,        // fp32 partial tiles summed in ring order
+    RMODE_RING_EPI = 1,    // the same, then the element-wise tail of Section 7.6
+    RMODE_BF16 = 2,        // 16-bit partial tiles (tail at run time)
+    RMODE_INPLACE = 3      // update in place: one fp32 accumulator per region (tail at run time)
+};
+
 // One reducer item: `rows` (8, 16 or 32) rows of the chunk starting at block row `row_in_block`.
-// chunk: the chunk's storage in slice 0 (fp32, or bf16 when partial_bf16); slice_stride in elements.
-// inplace: the chunk is the region's single fp32 accumulator (already the sum of all slices): read, clear, write Y.
-__device__ __forceinline__ void reduce_item(const void* __restrict__ chunk, size_t slice_stride, int partial_bf16,
+// chunk: the chunk's storage in slice 0 (fp32, or bf16 for RMODE_BF16); slice_stride in elements.
+// RMODE_INPLACE: the chunk is the region's single fp32 accumulator (already the sum of all slices): read,
+// clear, write Y.
+template <int RMODE>
+__device__ __forceinline__ void reduce_item(const void* __restrict__ chunk, size_t slice_stride,
                                             int row_in_block, int rows, void* Y, int M, int N, int R, int chunk_rows,
                                             int out_f32, int row_base, int col_base, int ncols_left, int lane,
-                                            const EpiOps& eo, int inplace, int l2_hints = 0) {
+                                            const EpiOps& eo, int l2_hints) {
     const int first = row_in_block >> 3;
     int end = (row_in_block + rows) >> 3;
     if (row_base + 8 * end > M) end = (M - row_base + 7) >> 3;     // the rest of the block is padding
-    if (inplace) {
+    if constexpr (RMODE == RMODE_INPLACE) {
         finish_item_inplace(static_cast<const float*>(chunk), first, end, Y, M, N, out_f32, row_base, col_base, ncols_left,
                             lane, eo);
-    } else if (partial_bf16) {
+    } else if constexpr (RMODE == RMODE_BF16) {
 #pragma unroll 1
         for (int rowsel = first; rowsel < end; ++rowsel)
             reduce_row_group_bf16<8>(static_cast<const __nv_bfloat16*>(chunk), slice_stride, rowsel, Y, M, N, R, chunk_rows,
@@ -458,8 +472,9 @@ __device__ __forceinline__ void reduce_item(const void* __restrict__ chunk, size
         const uint64_t pol_first = l2_policy_evict_first();
 #pragma unroll 1
         for (int rowsel = first; rowsel < end; ++rowsel)
-            reduce_row_group<8>(static_cast<const float*>(chunk), slice_stride, rowsel, Y, M, N, R, chunk_rows, out_f32,
-                                row_base, col_base, ncols_left, lane, eo, last_use, pol_first);
+            reduce_row_group<8, RMODE == RMODE_RING_EPI>(static_cast<const float*>(chunk), slice_stride, rowsel, Y, M, N, R,
+                                                         chunk_rows, out_f32, row_base, col_base, ncols_left, lane, eo,
+                                                         last_use, pol_first);
     }
 }
 
@@ -532,9 +547,10 @@ __device__ __forceinline__ void epi_store_frag_bf16(const uint32_t (&lo)[16], co
 // ---------------------------------------------------------------------------
 // fused persistent kernel
 // ---------------------------------------------------------------------------
-template <int CLUSTER>
+template <int CLUSTER, int RMODE>
 __global__ void __cluster_dims__(CLUSTER, 1, 1) __launch_bounds__(NUM_THREADS, 1)
 t3_fused_kernel(const __grid_constant__ KParams p) {
+    constexpr bool INPLACE = RMODE == RMODE_INPLACE, PARTIAL_BF16 = RMODE == RMODE_BF16;
     static_assert(CLUSTER == 2 || CLUSTER == 4, "one or two CTA pairs per cluster");
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) uint64_t bar_full[MAX_STAGES];    // leader's: both CTAs' loads of a stage landed
@@ -757,7 +773,7 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
         // Each warp owns 32 accumulator rows and walks them in 32-column chunks; the TMEM load of the
         // next chunk is in flight while the current one is transposed and stored.
         const int q = warp & 3;                                  // TMEM lane quarter this warp may read
-        const bool hint_st = (p.l2_hints & 12) != 0 && !p.partial_bf16 && !p.inplace;
+        const bool hint_st = (p.l2_hints & 12) != 0 && !PARTIAL_BF16 && !INPLACE;
         const uint64_t pol_st = (p.l2_hints & 4) ? l2_policy_evict_last() : l2_policy_evict_first();
         const uint32_t tempty0 = mapa_cluster(smem_u32(&bar_tempty[0]), lead);   // the pair leader's
         int jl = 0, acc = 0;
@@ -821,7 +837,7 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
             // this warp's row block (half * 4 + q) of slice r's tile in the region's slot
             const int slot = p.ring_slots > 0 ? seq % p.ring_slots : mt * p.sched.n_nt + nt;
             const size_t dst_off = static_cast<size_t>(slot) * static_cast<size_t>(p.slot_elems) +
-                                   static_cast<size_t>(p.inplace ? 0 : r) * static_cast<size_t>(p.tile_elems) +
+                                   static_cast<size_t>(INPLACE ? 0 : r) * static_cast<size_t>(p.tile_elems) +
                                    static_cast<size_t>((static_cast<int>(half) * EPI_WARPS + q) * p.sched.nc) * FRAG_ELEMS;
             float* dst = p.partials + dst_off;
             __nv_bfloat16* dst16 = reinterpret_cast<__nv_bfloat16*>(p.partials) + dst_off;
@@ -843,9 +859,9 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                     __syncwarp();
                     if (lane == 0) mbar_arrive_cluster_relaxed(tempty0 + static_cast<uint32_t>(acc) * 8u);
                 }
-                if (p.inplace) epi_red_frag(alo, ahi, lane, dst + ci * FRAG_ELEMS);
+                if constexpr (INPLACE) epi_red_frag(alo, ahi, lane, dst + ci * FRAG_ELEMS);
+                else if constexpr (PARTIAL_BF16) epi_store_frag_bf16(alo, ahi, lane, dst16 + ci * FRAG_ELEMS);
                 else if (hint_st) epi_store_frag_hint(alo, ahi, lane, dst + ci * FRAG_ELEMS, pol_st);
-                else if (p.partial_bf16) epi_store_frag_bf16(alo, ahi, lane, dst16 + ci * FRAG_ELEMS);
                 else epi_store_frag(alo, ahi, lane, dst + ci * FRAG_ELEMS);
                 if (ci + 1 < nchunks) {
                     tmem_ld_wait();
@@ -857,9 +873,9 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                         __syncwarp();
                         if (lane == 0) mbar_arrive_cluster_relaxed(tempty0 + static_cast<uint32_t>(acc) * 8u);
                     }
-                    if (p.inplace) epi_red_frag(blo, bhi, lane, dst + (ci + 1) * FRAG_ELEMS);
+                    if constexpr (INPLACE) epi_red_frag(blo, bhi, lane, dst + (ci + 1) * FRAG_ELEMS);
+                    else if constexpr (PARTIAL_BF16) epi_store_frag_bf16(blo, bhi, lane, dst16 + (ci + 1) * FRAG_ELEMS);
                     else if (hint_st) epi_store_frag_hint(blo, bhi, lane, dst + (ci + 1) * FRAG_ELEMS, pol_st);
-                    else if (p.partial_bf16) epi_store_frag_bf16(blo, bhi, lane, dst16 + (ci + 1) * FRAG_ELEMS);
                     else epi_store_frag(blo, bhi, lane, dst + (ci + 1) * FRAG_ELEMS);
                 }
             }
@@ -899,11 +915,11 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
                 const int slot = p.ring_slots > 0 ? seq % p.ring_slots : region;
                 const size_t chunk_off = static_cast<size_t>(slot) * static_cast<size_t>(p.slot_elems) +
                                          static_cast<size_t>(rb * p.sched.nc + cc) * FRAG_ELEMS;
-                const void* chunk = p.partial_bf16
+                const void* chunk = PARTIAL_BF16
                                         ? static_cast<const void*>(reinterpret_cast<const __nv_bfloat16*>(p.partials) + chunk_off)
                                         : static_cast<const void*>(p.partials + chunk_off);
-                reduce_item(chunk, static_cast<size_t>(p.tile_elems), p.partial_bf16, rib, p.sched.reduce_rows, p.Y, p.M, p.N,
-                            p.R, p.chunk_rows, p.out_f32, row_base, col_base, ncols_left, lane, p.epi, p.inplace, p.l2_hints);
+                reduce_item<RMODE>(chunk, static_cast<size_t>(p.tile_elems), rib, p.sched.reduce_rows, p.Y, p.M, p.N,
+                                   p.R, p.chunk_rows, p.out_f32, row_base, col_base, ncols_left, lane, p.epi, p.l2_hints);
                 if (p.ring_slots > 0) {
                     // every lane's loads of this item have returned (their values were used above)
                     __syncwarp();
@@ -956,11 +972,11 @@ t3_fused_kernel(const __grid_constant__ KParams p) {
 // ---------------------------------------------------------------------------
 // sequential baseline: the separate reduce kernel over full partial buffers (slot = region index)
 // ---------------------------------------------------------------------------
-template <int PARTIAL_BF16>       // compiled once per storage type, so that each keeps two blocks per SM
+template <int RMODE>       // compiled once per reducer mode, so that each keeps two blocks per SM
 __global__ void __launch_bounds__(256, 2) t3_reduce_kernel(const float* __restrict__ partials, void* Y, int M, int N, int R,
                                                            int chunk_rows, int out_f32, int BN, Sched sched,
-                                                           long long slot_elems, int tile_elems, EpiOps epi, int inplace) {
-    constexpr int partial_bf16 = PARTIAL_BF16;
+                                                           long long slot_elems, int tile_elems, EpiOps epi) {
+    constexpr bool partial_bf16 = RMODE == RMODE_BF16;
     const int lane = static_cast<int>(threadIdx.x) & 31;
     const long long warps = static_cast<long long>(gridDim.x) * (blockDim.x >> 5);
     const long long n_items = static_cast<long long>(sched.n_regions) * sched.items;
@@ -978,8 +994,8 @@ __global__ void __launch_bounds__(256, 2) t3_reduce_kernel(const float* __restri
                                  static_cast<size_t>(rb * sched.nc + cc) * FRAG_ELEMS;
         const void* chunk = partial_bf16 ? static_cast<const void*>(reinterpret_cast<const __nv_bfloat16*>(partials) + chunk_off)
                                          : static_cast<const void*>(partials + chunk_off);
-        reduce_item(chunk, static_cast<size_t>(tile_elems), partial_bf16, rib, sched.reduce_rows, Y, M, N, R, chunk_rows,
-                    out_f32, row_base, col_base, ncols_left, lane, epi, inplace);
+        reduce_item<RMODE>(chunk, static_cast<size_t>(tile_elems), rib, sched.reduce_rows, Y, M, N, R, chunk_rows,
+                           out_f32, row_base, col_base, ncols_left, lane, epi, 0);
     }
 }
 
