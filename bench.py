@@ -39,10 +39,10 @@ L2_FLUSH_BYTES = 512 << 20
 # ncu in an EARLIER, separate run (never measured inside this script): bytes per launch and the summary
 # under profiles/ that holds the capture's command and figures.  Absent: no capture for that workload.
 NCU_TRAFFIC = {
-    "C2_gpt2xl_fc2": (727.6e6, "profiles/t3_fused_kernel_C2.md"),
-    "C3b_megagpt_fc2": (1303.0e6, "profiles/t3_fused_kernel_C3b.md"),
-    # captured on the same shape scaled to M = 1 024 (1.609 GB per launch); traffic is proportional to M there
-    "C4_large_fc2": (4 * 1.609e9, "profiles/t3_fused_kernel_C4_scaled.md, x4 from the M = 1 024 capture"),
+    "C2_gpt2xl_fc2": (708.1e6, "profiles/t3_fused_kernel_C2.md"),
+    "C3b_megagpt_fc2": (1272.4e6, "profiles/t3_fused_kernel_C3b.md"),
+    # captured on the same shape scaled to M = 1 024 (1.555 GB per launch); traffic is proportional to M there
+    "C4_large_fc2": (4 * 1.555e9, "profiles/t3_fused_kernel_C4_scaled.md, x4 from the M = 1 024 capture"),
 }
 CHUNK_ARGS = ("tile_n", "group_tiles", "reducer_ctas", "reducer_warps", "reduce_rows", "stages", "ring_slots", "cluster_ctas",
               "partial_dtype", "order", "reduce", "split_k", "l2_hints")

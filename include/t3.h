@@ -126,7 +126,9 @@ typedef struct {
     int32_t mode;            /* t3_mode_t used by t3_gemm_rs                                         */
     int32_t tile_n;          /* output-tile width BN: multiple of 32 in [32,256]; 0 = auto           */
     int32_t group_tiles;     /* schedule group height in 256-row tiles (W reuse vs early trigger)    */
-    int32_t reducer_ctas;    /* CTAs (= SMs) that only reduce: the explicit SM split; 0 = none       */
+    int32_t reducer_ctas;    /* CTAs (= SMs) that only reduce: the explicit SM split; 0 = none, except */
+                             /* that SMs left without producer tiles (fewer tiles than CTA pairs) run  */
+                             /* reducers instead of idling                                             */
     int32_t reducer_warps;   /* reducer warps inside each GEMM CTA, 1..8; -1 = none; 0 = auto (8)    */
     int32_t reduce_rows;     /* rows of a reducer work item (a 32-column piece): 32, 16 or 8;        */
                              /* 0 = auto (16 when R > 8, else 32)                                    */
@@ -134,8 +136,10 @@ typedef struct {
     int32_t timeout_ms;      /* bound on every device-side wait; 0 = 1000                            */
     int32_t debug_flags;     /* T3_DEBUG_*                                                            */
     int32_t max_ctas;        /* cap on the persistent grid; 0 = one CTA per SM                       */
-    int32_t ring_slots;      /* fused mode: region slots in the recycled partial ring; 0 = auto,     */
-                             /* -1 = none (full partial buffers), else >= group_tiles               */
+    int32_t ring_slots;      /* fused mode: region slots in the recycled partial ring; 0 = auto (about */
+                             /* 64 MB, 40 MB for clusters of four on two-tile groups, never fewer than */
+                             /* the regions in flight), -1 = none (full partial buffers), else         */
+                             /* >= group_tiles                                                          */
     int32_t cluster_ctas;    /* CTAs per cluster: 2 (one CTA pair) or 4 (two pairs on vertically     */
                              /* adjacent tiles fetch each W k-block once for both; needs a library   */
                              /* built with the shared-fetch TMA file and an even number of 256-row   */
@@ -151,7 +155,8 @@ typedef struct {
                              /* reduce = T3_REDUCE_INPLACE when > 1; 0 = 1; at most 16 and at most    */
                              /* the slice's k-blocks.  For shapes with too few tiles to fill the GPU  */
                              /* (small M: the token-generation phase, Section 7.3).                  */
-    int32_t l2_hints;        /* L2 eviction-priority hints, a bit mask; 0 = auto (the measured default), */
+    int32_t l2_hints;        /* L2 eviction-priority hints, a bit mask; 0 = auto (3; 39 for clusters of  */
+                             /* four on two-tile groups, where a W tile has no reuse once fetched),     */
                              /* -1 = none.  1: X tiles are fetched evict_last; 2: reducers read partial */
                              /* tiles evict_first (their last use); 4 / 8: partial tiles are stored     */
                              /* evict_last / evict_first; 16 / 32: W tiles are fetched evict_last /     */
@@ -166,7 +171,7 @@ typedef struct {
     int32_t chunk_rows;        /* M / R: rows of one reduce-scatter chunk                    */
     int32_t tile_m, tile_n;    /* output tile = tracker region (Sec. 4.2.1 granularity)      */
     int32_t n_m_tiles, n_n_tiles;
-    int32_t n_jobs;            /* producer tiles: n_m_tiles * n_n_tiles * R                  */
+    int32_t n_jobs;            /* producer tiles: n_m_tiles * n_n_tiles * R * split_k        */
     int32_t n_regions;         /* tracked regions = output tiles                             */
     int32_t expected;          /* tracker threshold per region (landed 128-row half tiles)   */
     int32_t group_tiles;
