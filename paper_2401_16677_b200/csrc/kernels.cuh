@@ -9,6 +9,9 @@
 // MMAs for both, and each CTA's 128 accumulator rows land in its own TMEM,
 // drained by its own epilogue warps.
 //
+// The kernel is compiled once per cluster size and per reducer mode (RMode: how a region's stored tiles
+// become Y), so that every instantiation holds exactly one variant of the reducers' inner loop.
+//
 // CLUSTER = 2: one pair per cluster, every CTA fetches its own operands.
 // CLUSTER = 4 (built only when the file with the shared-fetch TMA wrapper is
 // present): two pairs per cluster work on vertically adjacent tiles (same W
@@ -77,12 +80,13 @@ struct alignas(64) KParams {
                             // > 0: the region with sequence number q uses slot q % ring_slots
     long long slot_elems;   // R * tile_elems: a slot holds the R partial tiles of one region
     int tile_elems;         // ROW_BLOCKS * nc * FRAG_ELEMS
-    int partial_bf16;       // 1: partial tiles are stored as bf16 (one rounding per slice), summed in fp32
+    int partial_bf16;       // 1: partial tiles are stored as bf16 (one rounding per slice), summed in fp32 (the host
+                            // launches the RMODE_BF16 instantiation; device code looks at its template argument)
     int w_kn;               // 1: W is stored [K][N] (N contiguous): the B operand is MN-major in shared memory
     void* Y;                // [M][N] bf16 or fp32
     uint32_t* counters;     // [n_regions] tracker: landed half tiles per region
     uint32_t* done;         // [n_regions] reduced items per region (frees the region's ring slot)
-    uint32_t* ctl;          // [0] reducer ticket, [1] CTAs done
+    uint32_t* ctl;          // [0] reducer ticket, [1] CTAs done, [2] epoch of the launch that is aborting
     int32_t* status;        // [4] code, where, block, detail
     int M, N, R, chunk_rows;
     int BN;
@@ -104,6 +108,7 @@ struct alignas(64) KParams {
     int inplace;            // 1: update-in-place reduction (Section 4.3's analog): the epilogues add every slice's
                             // tile into ONE fp32 accumulator tile per region with L2 reductions; the tracker then
                             // gates only the final convert / store pass, which also clears the accumulator
+                            // (the host launches the RMODE_INPLACE instantiation)
     int l2_hints;           // L2 eviction priorities: bit 0: X tiles fetched evict_last; bit 1: reducers read partial
                             // tiles evict_first (their last use); bit 2 / 3: partial tiles stored evict_last /
                             // evict_first; bit 4 / 5: W tiles fetched evict_last / evict_first
