@@ -462,6 +462,11 @@ int64_t t3_reduce_schedule(int64_t M, int64_t N, int64_t K, int32_t R, t3_dtype_
  * order[s] = (c - 1 - s) mod R, ending at c.  `order` has room for R ints. */
 int t3_ring_order(int32_t c, int32_t R, int32_t *order /* host */);
 
+/* Host-only: sizeof of the public structs in the order t3_chunking_t, t3_info_t, t3_status_t,
+ * t3_epilogue_t, t3_timeline_t, t3_tune_t, written to sizes[0..n) (n <= 6); returns how many exist (6).
+ * Lets a foreign-language binding check its struct definitions against the library it loaded. */
+int t3_abi_sizes(int32_t *sizes /* host */, int32_t n);
+
 int t3_last_error(void);               /* thread-local code of the last failed call */
 const char *t3_strerror(int code);     /* static string                              */
 int t3_version(void);

@@ -694,6 +694,14 @@ int run_mode(t3_plan_t pl, const Geometry& g, int mode, void* Y, cudaStream_t st
 extern "C" {
 
 int t3_version(void) { return T3_VERSION; }
+
+int t3_abi_sizes(int32_t* sizes, int32_t n) {
+    const int32_t all[6] = {static_cast<int32_t>(sizeof(t3_chunking_t)), static_cast<int32_t>(sizeof(t3_info_t)),
+                            static_cast<int32_t>(sizeof(t3_status_t)),   static_cast<int32_t>(sizeof(t3_epilogue_t)),
+                            static_cast<int32_t>(sizeof(t3_timeline_t)), static_cast<int32_t>(sizeof(t3_tune_t))};
+    for (int i = 0; sizes && i < n && i < 6; ++i) sizes[i] = all[i];
+    return 6;
+}
 int t3_shared_fetch_available(void) { return HAVE_SHARED_FETCH ? 1 : 0; }
 int t3_last_error(void) { return g_last_error; }
 

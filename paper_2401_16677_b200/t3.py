@@ -65,7 +65,7 @@ EXPORTS = [
     "t3_plan", "t3_gemm_rs", "t3_gemm_rs_mode", "t3_gemm_rs_ex", "t3_gemm_rs_host", "t3_gemm_rs_static", "t3_destroy",
     "t3_plan_info", "t3_plan_status", "t3_plan_tune", "t3_plan_timeline",
     "t3_plan_partials", "t3_plan_ring", "t3_plan_export_partials", "t3_geometry", "t3_schedule", "t3_reduce_schedule", "t3_ring_order",
-    "t3_last_error", "t3_strerror", "t3_version", "t3_shared_fetch_available",
+    "t3_last_error", "t3_strerror", "t3_version", "t3_shared_fetch_available", "t3_abi_sizes",
 ]
 
 
@@ -196,6 +196,13 @@ def lib() -> ctypes.CDLL:
         L.t3_last_error.restype = ctypes.c_int
         L.t3_strerror.argtypes = [ctypes.c_int]
         L.t3_strerror.restype = ctypes.c_char_p
+        L.t3_abi_sizes.argtypes = [ctypes.POINTER(ctypes.c_int32), i32]
+        L.t3_abi_sizes.restype = ctypes.c_int
+        sizes = (ctypes.c_int32 * 6)()
+        L.t3_abi_sizes(sizes, 6)
+        mine = [ctypes.sizeof(c) for c in (Chunking, Info, Status, Epilogue, Timeline, Tune)]
+        if list(sizes) != mine:
+            raise RuntimeError(f"{LIB_PATH}: struct sizes {list(sizes)} differ from this binding's {mine} (stale library?)")
         L.t3_version.restype = ctypes.c_int
         L.t3_shared_fetch_available.restype = ctypes.c_int
         _lib = L
